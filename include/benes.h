@@ -1,0 +1,131 @@
+/*
+ * benes.h -- C ABI of the B200 (sm_100a) Benes-network routing library.
+ *
+ * Problem statement (the build contract; the mounted paper has no passage on
+ * it): a rearrangeable Benes network of N = 2^n inputs has 2n-1 stages of N/2
+ * two-by-two switches.  benes_route computes the switch settings that make it
+ * realise a permutation pi given in GATHER form, out[j] = in[pi[j]];
+ * benes_apply pushes a payload through the stages.
+ *
+ * Canonical result.  Several settings realise the same pi; the library returns
+ * the one in which, at every recursion level and in every sub-network, the
+ * smallest output index of each constraint loop is served by the UPPER
+ * half-size sub-network.  The result is therefore unique and is compared
+ * bit for bit with the CPU oracle.
+ *
+ * Switch-bit layout (all entry points).  Stage-major.  A stage has
+ * W = max(1, N/64) 32-bit words; switch w of a stage is bit (w & 31) of word
+ * (w >> 5); 0 = straight, 1 = cross; unused bits are 0.  Recursion level l
+ * (0 <= l <= n-1) consists of 2^l sub-networks ("blocks") of size M = N >> l,
+ * block b owning flat positions [bM, (b+1)M) and, in every stage it owns,
+ * switches [b*M/2, (b+1)*M/2).  Stage l <= n-2 is the input side of level l,
+ * stage n-1 the middle, stage 2n-2-l the output side of level l.  Wiring: on
+ * the input side, switch s of a block sends its upper output to position s of
+ * the block's upper half and its lower output to position s of the lower
+ * half; the output side is the mirror image.  A batch is `batch` such
+ * records back to back: batch x (2n-1) x W words.
+ *
+ * Conventions.  Every pointer is a DEVICE pointer unless the name says
+ * "_host".  The caller owns every buffer it passes; the library owns only its
+ * internal workspace (one per device, grown on demand with cudaMalloc on the
+ * first call that needs it, or supplied by the caller).  Work is enqueued on
+ * `stream` and the call returns without synchronising, except where stated.
+ * Argument errors are detected on the host before anything is enqueued.
+ * Nothing throws, aborts or traps.  The library is not re-entrant: calls that
+ * share the workspace must be ordered (same stream, or externally
+ * synchronised).
+ */
+#ifndef BENES_H_
+#define BENES_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct CUstream_st *benes_stream_t; /* a cudaStream_t; NULL = default stream */
+
+enum {
+    BENES_OK = 0,
+    BENES_ERR_BADARG = -1,          /* null pointer, log2n or batch out of range, bad elem_bytes */
+    BENES_ERR_CUDA = -2,            /* a CUDA runtime call or launch failed */
+    BENES_ERR_NOMEM = -3,           /* workspace could not be allocated / supplied one too small */
+    BENES_ERR_NOT_PERMUTATION = -4  /* benes_validate_perm only */
+};
+
+#define BENES_MAX_LOG2N 30
+
+/*
+ * Switch settings (steps: inverse scatter, successor pairing, pointer-jumping
+ * loop labelling to the minimum index, 2-colouring, first/last stage,
+ * sub-permutation compaction; all n levels).
+ *   perm        : batch x N uint32, each row a permutation of [0, N); read only.
+ *   log2n       : 1 .. BENES_MAX_LOG2N.
+ *   batch       : >= 1 independent permutations.
+ *   switch_bits : batch x (2n-1) x W words (benes_switch_words), fully overwritten.
+ * If a row is not a permutation the result is unspecified but every access
+ * stays in bounds.  Returns BENES_OK or a negative status.
+ */
+int benes_route(const uint32_t *perm, int log2n, int batch, uint32_t *switch_bits,
+                benes_stream_t stream);
+
+/*
+ * Route a payload of 4-byte elements through the network, one pass per stage:
+ * out[b][j] = in[b][pi_b[j]] when switch_bits came from benes_route(pi).
+ *   in, out : batch x N elements; must not overlap; in is read only.
+ */
+int benes_apply(const uint32_t *switch_bits, const void *in, void *out, int log2n, int batch,
+                benes_stream_t stream);
+
+/* Same with an explicit element size: elem_bytes must be 4 or 8. */
+int benes_apply_ex(const uint32_t *switch_bits, const void *in, void *out, int elem_bytes,
+                   int log2n, int batch, benes_stream_t stream);
+
+/*
+ * Host-buffer variants: copy the inputs to the device, run, copy the result
+ * back and SYNCHRONISE `stream` before returning.  Buffers are ordinary or
+ * pinned host memory.  Device staging lives in the library workspace.
+ */
+int benes_route_host(const uint32_t *perm_host, int log2n, int batch, uint32_t *switch_bits_host,
+                     benes_stream_t stream);
+int benes_apply_host(const uint32_t *switch_bits_host, const void *in_host, void *out_host,
+                     int elem_bytes, int log2n, int batch, benes_stream_t stream);
+
+/* Number of 32-bit words of switch_bits for (log2n, batch); 0 on bad arguments. */
+size_t benes_switch_words(int log2n, int batch);
+
+/* Scratch bytes benes_route / benes_apply_ex need for these arguments. */
+size_t benes_route_workspace_bytes(int log2n, int batch);
+size_t benes_apply_workspace_bytes(int elem_bytes, int log2n, int batch);
+
+/*
+ * Hand the library a caller-owned device scratch buffer (256-byte aligned) to
+ * use instead of its own; pass (NULL, 0) to return to the internal one.  With
+ * a caller buffer no entry point allocates; a call that needs more than
+ * `bytes` fails with BENES_ERR_NOMEM.
+ */
+int benes_set_workspace(void *dev_ptr, size_t bytes);
+
+/* Free the internal workspace of the current device (synchronises the device). */
+int benes_release_workspace(void);
+
+/*
+ * Check that every row of perm is a permutation of [0, N).  Synchronises
+ * `stream`.  Returns BENES_OK, BENES_ERR_NOT_PERMUTATION or another error.
+ */
+int benes_validate_perm(const uint32_t *perm, int log2n, int batch, benes_stream_t stream);
+
+/* Kernels launched by this library in this process so far (host-side counter). */
+unsigned long long benes_launch_count(void);
+
+/* Largest block size (log2) finished inside one CTA by the fused kernel. */
+int benes_fused_log2m(void);
+
+const char *benes_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BENES_H_ */

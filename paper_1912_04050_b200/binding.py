@@ -1,0 +1,193 @@
+"""ctypes binding of ``libbenes.so`` -- argument marshalling only.
+
+Function names and argument orders are those of ``include/benes.h``.  Device
+buffers are ``torch`` CUDA tensors (PyTorch is used for device memory and
+streams, nothing else); every step of the path runs inside the library's CUDA
+kernels.  There is no CPU fallback: if the library has not been built, loading
+raises ``RuntimeError``.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libbenes.so")
+
+BENES_OK = 0
+BENES_ERR_BADARG = -1
+BENES_ERR_CUDA = -2
+BENES_ERR_NOMEM = -3
+BENES_ERR_NOT_PERMUTATION = -4
+
+# every symbol include/benes.h declares: name -> (restype, argtypes)
+_vp, _i, _sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+SYMBOLS = {
+    "benes_route": (_i, [_vp, _i, _i, _vp, _vp]),
+    "benes_apply": (_i, [_vp, _vp, _vp, _i, _i, _vp]),
+    "benes_apply_ex": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp]),
+    "benes_route_host": (_i, [_vp, _i, _i, _vp, _vp]),
+    "benes_apply_host": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp]),
+    "benes_switch_words": (_sz, [_i, _i]),
+    "benes_route_workspace_bytes": (_sz, [_i, _i]),
+    "benes_apply_workspace_bytes": (_sz, [_i, _i, _i]),
+    "benes_set_workspace": (_i, [_vp, _sz]),
+    "benes_release_workspace": (_i, []),
+    "benes_validate_perm": (_i, [_vp, _i, _i, _vp]),
+    "benes_launch_count": (ctypes.c_ulonglong, []),
+    "benes_fused_log2m": (_i, []),
+    "benes_status_string": (ctypes.c_char_p, [_i]),
+}
+
+_lib = None
+
+
+class BenesError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        super().__init__("%s failed: %s (%d)" % (what, status_string(status), status))
+
+
+def load() -> ctypes.CDLL:
+    """Load the CUDA library; fails loudly if it is not built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                "libbenes.so is not built (%s); run `python -m paper_1912_04050_b200.build`. "
+                "There is no CPU fallback." % LIB_PATH)
+        lib = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in SYMBOLS.items():
+            fn = getattr(lib, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = lib
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return load().benes_status_string(status).decode()
+
+
+def _check(status: int, what: str) -> None:
+    if status != BENES_OK:
+        raise BenesError(status, what)
+
+
+def _dev_ptr(t: torch.Tensor, what: str) -> int:
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.is_contiguous()):
+        raise TypeError("%s must be a contiguous CUDA tensor" % what)
+    return t.data_ptr()
+
+
+def _host_ptr(t, what: str) -> int:
+    if isinstance(t, torch.Tensor):
+        if t.is_cuda or not t.is_contiguous():
+            raise TypeError("%s must be a contiguous host tensor" % what)
+        return t.data_ptr()
+    return t.ctypes.data        # numpy array
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def benes_switch_words(log2n: int, batch: int) -> int:
+    return load().benes_switch_words(log2n, batch)
+
+
+def benes_route_workspace_bytes(log2n: int, batch: int) -> int:
+    return load().benes_route_workspace_bytes(log2n, batch)
+
+
+def benes_apply_workspace_bytes(elem_bytes: int, log2n: int, batch: int) -> int:
+    return load().benes_apply_workspace_bytes(elem_bytes, log2n, batch)
+
+
+def benes_route(perm: torch.Tensor, log2n: int, batch: int, switch_bits: torch.Tensor, stream=None) -> None:
+    _check(load().benes_route(_dev_ptr(perm, "perm"), log2n, batch,
+                              _dev_ptr(switch_bits, "switch_bits"), _stream(stream)), "benes_route")
+
+
+def benes_apply(switch_bits: torch.Tensor, inp: torch.Tensor, out: torch.Tensor, log2n: int, batch: int,
+                stream=None) -> None:
+    _check(load().benes_apply(_dev_ptr(switch_bits, "switch_bits"), _dev_ptr(inp, "in"),
+                              _dev_ptr(out, "out"), log2n, batch, _stream(stream)), "benes_apply")
+
+
+def benes_apply_ex(switch_bits: torch.Tensor, inp: torch.Tensor, out: torch.Tensor, elem_bytes: int,
+                   log2n: int, batch: int, stream=None) -> None:
+    _check(load().benes_apply_ex(_dev_ptr(switch_bits, "switch_bits"), _dev_ptr(inp, "in"),
+                                 _dev_ptr(out, "out"), elem_bytes, log2n, batch, _stream(stream)),
+           "benes_apply_ex")
+
+
+def benes_route_host(perm_host, log2n: int, batch: int, switch_bits_host, stream=None) -> None:
+    _check(load().benes_route_host(_host_ptr(perm_host, "perm_host"), log2n, batch,
+                                   _host_ptr(switch_bits_host, "switch_bits_host"), _stream(stream)),
+           "benes_route_host")
+
+
+def benes_apply_host(switch_bits_host, in_host, out_host, elem_bytes: int, log2n: int, batch: int,
+                     stream=None) -> None:
+    _check(load().benes_apply_host(_host_ptr(switch_bits_host, "switch_bits_host"),
+                                   _host_ptr(in_host, "in_host"), _host_ptr(out_host, "out_host"),
+                                   elem_bytes, log2n, batch, _stream(stream)), "benes_apply_host")
+
+
+def benes_set_workspace(buf, nbytes: int = 0) -> None:
+    if buf is None:
+        _check(load().benes_set_workspace(None, 0), "benes_set_workspace")
+    else:
+        _check(load().benes_set_workspace(_dev_ptr(buf, "workspace"),
+                                          nbytes or buf.numel() * buf.element_size()),
+               "benes_set_workspace")
+
+
+def benes_release_workspace() -> None:
+    _check(load().benes_release_workspace(), "benes_release_workspace")
+
+
+def benes_validate_perm(perm: torch.Tensor, log2n: int, batch: int, stream=None) -> bool:
+    """True if every row is a permutation; False if not; raises on other errors."""
+    rc = load().benes_validate_perm(_dev_ptr(perm, "perm"), log2n, batch, _stream(stream))
+    if rc == BENES_ERR_NOT_PERMUTATION:
+        return False
+    _check(rc, "benes_validate_perm")
+    return True
+
+
+def benes_launch_count() -> int:
+    return load().benes_launch_count()
+
+
+def benes_fused_log2m() -> int:
+    return load().benes_fused_log2m()
+
+
+# ---- small conveniences that only allocate outputs -------------------------------------------
+def route(perm: torch.Tensor, stream=None) -> torch.Tensor:
+    """perm: (N,) or (batch, N) CUDA tensor holding uint32 values (dtype int32 or uint32).
+    Returns the switch bits as an int32 tensor of shape ([batch,] 2n-1, W)."""
+    N = perm.shape[-1]
+    log2n = N.bit_length() - 1
+    if N < 2 or (1 << log2n) != N:
+        raise ValueError("N must be a power of two >= 2")
+    batch = perm.numel() // N
+    W = max(1, N // 64)
+    bits = torch.empty(perm.shape[:-1] + (2 * log2n - 1, W), dtype=torch.int32, device=perm.device)
+    benes_route(perm, log2n, batch, bits, stream)
+    return bits
+
+
+def apply(switch_bits: torch.Tensor, x: torch.Tensor, stream=None) -> torch.Tensor:
+    """Push payload x ((N,) or (batch, N), 4- or 8-byte dtype) through the network."""
+    N = x.shape[-1]
+    log2n = N.bit_length() - 1
+    batch = x.numel() // N
+    out = torch.empty_like(x)
+    benes_apply_ex(switch_bits, x, out, x.element_size(), log2n, batch, stream)
+    return out

@@ -1,0 +1,299 @@
+// extern "C" entry points (declared in include/benes.h), argument checks,
+// workspace management and the host-side level loop.
+#include "common.cuh"
+
+#include <mutex>
+
+namespace benes {
+namespace {
+
+constexpr int kMaxDevices = 64;
+constexpr size_t kAlign = 256;
+// Flat elements processed together by the per-level path (indices are 32 bit).
+constexpr size_t kMaxFlat = size_t(1) << 30;
+
+struct Workspace {
+    void *own = nullptr;       // library-owned buffer
+    size_t own_bytes = 0;
+    void *user = nullptr;      // caller-owned buffer (takes precedence)
+    size_t user_bytes = 0;
+};
+
+Workspace g_ws[kMaxDevices];
+std::mutex g_mu;
+
+inline size_t align_up(size_t v) { return (v + kAlign - 1) & ~(kAlign - 1); }
+
+// Returns a device scratch buffer of at least `bytes`.
+int get_workspace(size_t bytes, void **out) {
+    int dev = 0;
+    BENES_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return BENES_ERR_CUDA;
+    std::lock_guard<std::mutex> lk(g_mu);
+    Workspace &w = g_ws[dev];
+    if (w.user) {
+        if (bytes > w.user_bytes) return BENES_ERR_NOMEM;
+        *out = w.user;
+        return BENES_OK;
+    }
+    if (bytes > w.own_bytes) {
+        if (w.own) {
+            BENES_CUDA_TRY(cudaDeviceSynchronize());
+            cudaFree(w.own);
+            w.own = nullptr;
+            w.own_bytes = 0;
+        }
+        if (cudaMalloc(&w.own, bytes) != cudaSuccess) {
+            cudaGetLastError();
+            w.own = nullptr;
+            return BENES_ERR_NOMEM;
+        }
+        w.own_bytes = bytes;
+    }
+    *out = w.own;
+    return BENES_OK;
+}
+
+inline bool bad_shape(int log2n, int batch) {
+    return log2n < 1 || log2n > BENES_MAX_LOG2N || batch < 1;
+}
+
+inline size_t stage_words(int log2n) { return log2n >= 6 ? (size_t(1) << (log2n - 6)) : 1; }
+
+// permutations per chunk of the per-level path
+inline size_t level_chunk(int log2n, size_t batch) {
+    size_t per = kMaxFlat >> log2n;
+    if (per < 1) per = 1;
+    return batch < per ? batch : per;
+}
+
+size_t route_ws_bytes(int log2n, size_t batch) {
+    if (log2n <= kFusedLog2M) return 0;
+    size_t T = level_chunk(log2n, batch) << log2n;
+    // Pa, Pb, Qa, Qb (uint32) + words (uint64)
+    return 4 * align_up(T * 4) + align_up(T * 8);
+}
+
+size_t apply_ws_bytes(int elem_bytes, int log2n, size_t batch) {
+    if (log2n < 2) return 0;
+    return align_up((batch << log2n) * size_t(elem_bytes));
+}
+
+// Levels 0 .. n-kFusedLog2M-1 in HBM, then the fused tail.
+int route_levels(const uint32_t *perm, int n, size_t batch, uint32_t *bits, char *ws, cudaStream_t s) {
+    const size_t T = batch << n;
+    uint32_t *Pbuf[2], *Qbuf[2];
+    size_t off = 0;
+    Pbuf[0] = reinterpret_cast<uint32_t *>(ws + off); off += align_up(T * 4);
+    Pbuf[1] = reinterpret_cast<uint32_t *>(ws + off); off += align_up(T * 4);
+    Qbuf[0] = reinterpret_cast<uint32_t *>(ws + off); off += align_up(T * 4);
+    Qbuf[1] = reinterpret_cast<uint32_t *>(ws + off); off += align_up(T * 4);
+    unsigned long long *Wd = reinterpret_cast<unsigned long long *>(ws + off);
+
+    BitsLayout L{bits, n, n - 6};
+    const uint32_t *P = perm;
+    uint32_t *Q = Qbuf[0];
+    int rc = launch_inverse(P, Q, T, n, s);
+    if (rc) return rc;
+    int cur = 0;
+    for (int level = 0; n - level > kFusedLog2M; ++level) {
+        const int m = n - level;
+        if ((rc = launch_build(P, Q, Wd, T, m, s))) return rc;
+        for (int r = 1; r < m - 1; ++r)
+            if ((rc = launch_jump(Wd, T, s))) return rc;
+        if ((rc = launch_jump_last(Wd, T, L, 2 * n - 2 - level, s))) return rc;
+        uint32_t *Pn = Pbuf[cur], *Qn = Qbuf[cur ^ 1];
+        if ((rc = launch_split(P, Q, Pn, Qn, T, m, L, level, 2 * n - 2 - level, s))) return rc;
+        P = Pn;
+        Q = Qn;
+        cur ^= 1;
+    }
+    return launch_fused(P, T, kFusedLog2M, bits, n, s);
+}
+
+}  // namespace
+}  // namespace benes
+
+using namespace benes;
+
+extern "C" {
+
+size_t benes_switch_words(int log2n, int batch) {
+    if (bad_shape(log2n, batch)) return 0;
+    return size_t(batch) * size_t(2 * log2n - 1) * stage_words(log2n);
+}
+
+size_t benes_route_workspace_bytes(int log2n, int batch) {
+    if (bad_shape(log2n, batch)) return 0;
+    return route_ws_bytes(log2n, size_t(batch));
+}
+
+size_t benes_apply_workspace_bytes(int elem_bytes, int log2n, int batch) {
+    if (bad_shape(log2n, batch) || (elem_bytes != 4 && elem_bytes != 8)) return 0;
+    return apply_ws_bytes(elem_bytes, log2n, size_t(batch));
+}
+
+int benes_set_workspace(void *dev_ptr, size_t bytes) {
+    if ((dev_ptr == nullptr) != (bytes == 0)) return BENES_ERR_BADARG;
+    if (reinterpret_cast<uintptr_t>(dev_ptr) % kAlign) return BENES_ERR_BADARG;
+    int dev = 0;
+    BENES_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return BENES_ERR_CUDA;
+    std::lock_guard<std::mutex> lk(g_mu);
+    g_ws[dev].user = dev_ptr;
+    g_ws[dev].user_bytes = bytes;
+    return BENES_OK;
+}
+
+int benes_release_workspace(void) {
+    int dev = 0;
+    BENES_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return BENES_ERR_CUDA;
+    std::lock_guard<std::mutex> lk(g_mu);
+    Workspace &w = g_ws[dev];
+    if (w.own) {
+        BENES_CUDA_TRY(cudaDeviceSynchronize());
+        BENES_CUDA_TRY(cudaFree(w.own));
+        w.own = nullptr;
+        w.own_bytes = 0;
+    }
+    return BENES_OK;
+}
+
+int benes_route(const uint32_t *perm, int log2n, int batch, uint32_t *switch_bits,
+                benes_stream_t stream) {
+    if (!perm || !switch_bits || bad_shape(log2n, batch)) return BENES_ERR_BADARG;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    const int n = log2n;
+    if (n <= kFusedLog2M) {
+        // whole permutations fit one CTA each
+        const size_t max_ctas = size_t(1) << 30;
+        for (size_t b0 = 0; b0 < size_t(batch); b0 += max_ctas) {
+            size_t nb = size_t(batch) - b0 < max_ctas ? size_t(batch) - b0 : max_ctas;
+            int rc = launch_fused(perm + (b0 << n), nb << n, n,
+                                  switch_bits + b0 * size_t(2 * n - 1) * stage_words(n), n, s);
+            if (rc) return rc;
+        }
+        return BENES_OK;
+    }
+    void *ws = nullptr;
+    int rc = get_workspace(route_ws_bytes(n, size_t(batch)), &ws);
+    if (rc) return rc;
+    const size_t chunk = level_chunk(n, size_t(batch));
+    for (size_t b0 = 0; b0 < size_t(batch); b0 += chunk) {
+        size_t nb = size_t(batch) - b0 < chunk ? size_t(batch) - b0 : chunk;
+        rc = route_levels(perm + (b0 << n), n, nb,
+                          switch_bits + b0 * size_t(2 * n - 1) * stage_words(n),
+                          static_cast<char *>(ws), s);
+        if (rc) return rc;
+    }
+    return BENES_OK;
+}
+
+int benes_apply_ex(const uint32_t *switch_bits, const void *in, void *out, int elem_bytes,
+                   int log2n, int batch, benes_stream_t stream) {
+    if (!switch_bits || !in || !out || in == out || bad_shape(log2n, batch)) return BENES_ERR_BADARG;
+    if (elem_bytes != 4 && elem_bytes != 8) return BENES_ERR_BADARG;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    const int n = log2n;
+    const int stages = 2 * n - 1;
+    void *ws = nullptr;
+    if (n >= 2) {
+        int rc = get_workspace(apply_ws_bytes(elem_bytes, n, size_t(batch)), &ws);
+        if (rc) return rc;
+    }
+    // ping-pong between `out` and the scratch buffer so that the last stage lands in `out`
+    const void *src = in;
+    for (int st = 0; st < stages; ++st) {
+        void *dst = ((stages - 1 - st) % 2 == 0) ? out : ws;
+        int rc = launch_apply_stage(switch_bits, src, dst, elem_bytes, st, n, size_t(batch), s);
+        if (rc) return rc;
+        src = dst;
+    }
+    return BENES_OK;
+}
+
+int benes_apply(const uint32_t *switch_bits, const void *in, void *out, int log2n, int batch,
+                benes_stream_t stream) {
+    return benes_apply_ex(switch_bits, in, out, 4, log2n, batch, stream);
+}
+
+int benes_route_host(const uint32_t *perm_host, int log2n, int batch, uint32_t *switch_bits_host,
+                     benes_stream_t stream) {
+    if (!perm_host || !switch_bits_host || bad_shape(log2n, batch)) return BENES_ERR_BADARG;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    const size_t perm_bytes = (size_t(batch) << log2n) * 4;
+    const size_t bits_bytes = benes_switch_words(log2n, batch) * 4;
+    const size_t inner = route_ws_bytes(log2n, size_t(batch));
+    void *ws = nullptr;
+    int rc = get_workspace(align_up(inner) + align_up(perm_bytes) + align_up(bits_bytes), &ws);
+    if (rc) return rc;
+    char *base = static_cast<char *>(ws);
+    uint32_t *d_perm = reinterpret_cast<uint32_t *>(base + align_up(inner));
+    uint32_t *d_bits = reinterpret_cast<uint32_t *>(base + align_up(inner) + align_up(perm_bytes));
+    BENES_CUDA_TRY(cudaMemcpyAsync(d_perm, perm_host, perm_bytes, cudaMemcpyHostToDevice, s));
+    rc = benes_route(d_perm, log2n, batch, d_bits, stream);
+    if (rc) return rc;
+    BENES_CUDA_TRY(cudaMemcpyAsync(switch_bits_host, d_bits, bits_bytes, cudaMemcpyDeviceToHost, s));
+    BENES_CUDA_TRY(cudaStreamSynchronize(s));
+    return BENES_OK;
+}
+
+int benes_apply_host(const uint32_t *switch_bits_host, const void *in_host, void *out_host,
+                     int elem_bytes, int log2n, int batch, benes_stream_t stream) {
+    if (!switch_bits_host || !in_host || !out_host || bad_shape(log2n, batch)) return BENES_ERR_BADARG;
+    if (elem_bytes != 4 && elem_bytes != 8) return BENES_ERR_BADARG;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    const size_t data_bytes = (size_t(batch) << log2n) * size_t(elem_bytes);
+    const size_t bits_bytes = benes_switch_words(log2n, batch) * 4;
+    const size_t inner = apply_ws_bytes(elem_bytes, log2n, size_t(batch));
+    void *ws = nullptr;
+    int rc = get_workspace(align_up(inner) + 2 * align_up(data_bytes) + align_up(bits_bytes), &ws);
+    if (rc) return rc;
+    char *base = static_cast<char *>(ws);
+    char *d_in = base + align_up(inner);
+    char *d_out = d_in + align_up(data_bytes);
+    uint32_t *d_bits = reinterpret_cast<uint32_t *>(d_out + align_up(data_bytes));
+    BENES_CUDA_TRY(cudaMemcpyAsync(d_bits, switch_bits_host, bits_bytes, cudaMemcpyHostToDevice, s));
+    BENES_CUDA_TRY(cudaMemcpyAsync(d_in, in_host, data_bytes, cudaMemcpyHostToDevice, s));
+    rc = benes_apply_ex(d_bits, d_in, d_out, elem_bytes, log2n, batch, stream);
+    if (rc) return rc;
+    BENES_CUDA_TRY(cudaMemcpyAsync(out_host, d_out, data_bytes, cudaMemcpyDeviceToHost, s));
+    BENES_CUDA_TRY(cudaStreamSynchronize(s));
+    return BENES_OK;
+}
+
+int benes_validate_perm(const uint32_t *perm, int log2n, int batch, benes_stream_t stream) {
+    if (!perm || bad_shape(log2n, batch)) return BENES_ERR_BADARG;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    const size_t total = size_t(batch) << log2n;
+    const size_t seen_bytes = align_up(((total + 31) / 32) * 4);
+    void *ws = nullptr;
+    int rc = get_workspace(seen_bytes + kAlign, &ws);
+    if (rc) return rc;
+    uint32_t *seen = static_cast<uint32_t *>(ws);
+    uint32_t *flag = reinterpret_cast<uint32_t *>(static_cast<char *>(ws) + seen_bytes);
+    BENES_CUDA_TRY(cudaMemsetAsync(ws, 0, seen_bytes + kAlign, s));
+    if ((rc = launch_validate(perm, total, log2n, seen, flag, s))) return rc;
+    uint32_t h = 0;
+    BENES_CUDA_TRY(cudaMemcpyAsync(&h, flag, 4, cudaMemcpyDeviceToHost, s));
+    BENES_CUDA_TRY(cudaStreamSynchronize(s));
+    return h ? BENES_ERR_NOT_PERMUTATION : BENES_OK;
+}
+
+unsigned long long benes_launch_count(void) { return g_launches; }
+
+int benes_fused_log2m(void) { return kFusedLog2M; }
+
+const char *benes_status_string(int status) {
+    switch (status) {
+        case BENES_OK: return "ok";
+        case BENES_ERR_BADARG: return "bad argument";
+        case BENES_ERR_CUDA: return "CUDA runtime error";
+        case BENES_ERR_NOMEM: return "workspace allocation failed or caller workspace too small";
+        case BENES_ERR_NOT_PERMUTATION: return "input is not a permutation";
+        default: return "unknown status";
+    }
+}
+
+}  // extern "C"

@@ -91,11 +91,12 @@ def bit_reversal_perm(log2n: int) -> np.ndarray:
 
 
 def transpose_perm(log2n: int) -> np.ndarray:
-    """Index map of a square-matrix transpose: pi[r*S + c] = c*S + r, S = 2^(log2n/2)."""
-    assert log2n % 2 == 0
-    S = 1 << (log2n // 2)
+    """Index map of a matrix transpose: pi[r*C + c] = c*R + r for an R x C matrix,
+    R = 2^floor(log2n/2), C = N/R (square when log2n is even)."""
+    R = 1 << (log2n // 2)
+    C = (1 << log2n) // R
     j = np.arange(1 << log2n, dtype=np.uint32)
-    return ((j % S) * S + j // S).astype(np.uint32)
+    return ((j % C) * R + j // C).astype(np.uint32)
 
 
 def payload_f32(n_elems: int, seed: int) -> np.ndarray:

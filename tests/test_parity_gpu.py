@@ -1,0 +1,219 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU
+oracle on the same seeded inputs.  Integer / bit work: the bar is bit-exact."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_1912_04050_b200 import binding, build, inputs
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    build.build()
+    binding.load()
+    yield
+    binding.benes_release_workspace()
+
+
+def dev(a: np.ndarray) -> torch.Tensor:
+    """numpy (uint32/uint64/float32) -> CUDA tensor with the same bytes."""
+    view = {4: np.int32, 8: np.int64}[a.dtype.itemsize]
+    return torch.from_numpy(np.ascontiguousarray(a).view(view)).cuda()
+
+
+def host(t: torch.Tensor, dtype) -> np.ndarray:
+    return t.cpu().numpy().view(dtype)
+
+
+def gpu_route(perm: np.ndarray, n: int) -> np.ndarray:
+    p = dev(perm)
+    batch = perm.size >> n
+    bits = torch.full((binding.benes_switch_words(n, batch),), -1, dtype=torch.int32, device="cuda")
+    binding.benes_route(p, n, batch, bits)
+    torch.cuda.synchronize()
+    shape = (2 * n - 1, max(1, (1 << n) // 64))
+    return host(bits, np.uint32).reshape(((batch,) if perm.ndim == 2 else ()) + shape)
+
+
+def gpu_apply(bits: np.ndarray, x: np.ndarray, n: int) -> np.ndarray:
+    batch = x.size >> n
+    out = torch.empty_like(dev(x))
+    binding.benes_apply_ex(dev(bits), dev(x), out, x.dtype.itemsize, n, batch)
+    torch.cuda.synchronize()
+    return host(out, x.dtype).reshape(x.shape)
+
+
+# ---- route ------------------------------------------------------------------
+@pytest.mark.parametrize("n", list(range(1, 19)))
+def test_route_random_every_size(n):
+    """n = 1..13 run in one CTA; 14.. take 1.. HBM levels first, then the fused tail."""
+    perm = inputs.random_perm(n, 100 + n)
+    assert np.array_equal(gpu_route(perm, n), oracle.route(perm, n))
+
+
+@pytest.mark.parametrize("n,batch", [(1, 5), (2, 7), (3, 33), (5, 64), (6, 3), (8, 1000), (11, 5),
+                                     (13, 3), (14, 3), (15, 2), (16, 5)])
+def test_route_batched(n, batch):
+    perm = inputs.random_perm_batch(n, batch, seed0=7 * n)
+    assert np.array_equal(gpu_route(perm, n), oracle.route(perm, n))
+
+
+@pytest.mark.parametrize("n", [4, 10, 13, 14, 16, 18])
+@pytest.mark.parametrize("kind", ["identity", "shift1", "bitrev", "transpose", "sattolo"])
+def test_route_structured(n, kind):
+    perm = inputs.structured_perms(n)[kind]
+    assert np.array_equal(gpu_route(perm, n), oracle.route(perm, n))
+
+
+def test_route_exhaustive_n8():
+    """All 40320 permutations of N = 8 in one batched call."""
+    import itertools
+    perms = np.array(list(itertools.permutations(range(8))), dtype=np.uint32)
+    assert np.array_equal(gpu_route(perms, 3), oracle.route(perms, 3))
+
+
+# ---- apply ------------------------------------------------------------------
+@pytest.mark.parametrize("n", [1, 2, 3, 5, 6, 7, 10, 13, 16])
+@pytest.mark.parametrize("dtype", [np.uint32, np.uint64])
+def test_apply_random_settings(n, dtype):
+    """Arbitrary switch settings (not produced by route): checks wiring and layout alone."""
+    rng = np.random.default_rng(n)
+    batch = 3
+    W = max(1, (1 << n) // 64)
+    bits = rng.integers(0, 2 ** 32, size=(batch, 2 * n - 1, W), dtype=np.uint64).astype(np.uint32)
+    if n < 6:
+        bits &= np.uint32((1 << (1 << (n - 1))) - 1)
+    x = rng.integers(0, 2 ** 63, size=(batch, 1 << n), dtype=np.uint64).astype(dtype)
+    assert np.array_equal(gpu_apply(bits, x, n), oracle.apply(bits, x, n))
+
+
+def test_apply_does_not_touch_input():
+    n = 12
+    perm = inputs.random_perm(n, 1)
+    x = inputs.payload_u64(1 << n, 9)
+    dx = dev(x)
+    bits = dev(oracle.route(perm, n))
+    out = torch.empty_like(dx)
+    binding.benes_apply_ex(bits, dx, out, 8, n, 1)
+    torch.cuda.synchronize()
+    assert np.array_equal(host(dx, np.uint64), x)
+    assert np.array_equal(host(out, np.uint64), x[perm])
+
+
+# ---- the five configurations ------------------------------------------------------
+def test_config1_n1024_identity_payload():
+    n = 10
+    perm = inputs.random_perm(n, 0)
+    bits = gpu_route(perm, n)
+    assert bits.shape == (19, 16)
+    assert np.array_equal(bits, oracle.route(perm, n))
+    out = gpu_apply(bits, inputs.identity_perm(n), n)
+    assert np.array_equal(out, perm)
+    assert np.array_equal(out, oracle.apply(bits, inputs.identity_perm(n), n))
+
+
+def test_config2_batch_16384_of_256():
+    n, batch = 8, 16384
+    perm = inputs.random_perm_batch(n, batch, seed0=0)
+    bits = gpu_route(perm, n)
+    assert bits.shape == (batch, 15, 4)
+    assert np.array_equal(bits, oracle.route(perm, n))
+    ident = np.tile(inputs.identity_perm(n), (batch, 1))
+    assert np.array_equal(gpu_apply(bits, ident, n), perm)
+
+
+def test_config3_n2p20_fp32_payload():
+    n = 20
+    perm = inputs.random_perm(n, 1)
+    bits = gpu_route(perm, n)
+    assert np.array_equal(bits, oracle.route(perm, n))
+    x = inputs.payload_f32(1 << n, 1)
+    out = gpu_apply(bits, x, n)
+    assert np.array_equal(out.view(np.uint32), x[perm].view(np.uint32))
+    assert np.array_equal(out.view(np.uint32), oracle.apply(bits, x, n).view(np.uint32))
+
+
+@pytest.mark.parametrize("kind", ["identity", "shift1", "bitrev", "transpose", "sattolo"])
+def test_config5_structured_n2p24(kind):
+    n = 24
+    perm = inputs.structured_perms(n)[kind]
+    bits = gpu_route(perm, n)
+    assert np.array_equal(bits, oracle.route(perm, n))
+    assert np.array_equal(gpu_apply(bits, inputs.identity_perm(n), n), perm)
+
+
+def test_config4_n2p26_u64_payload():
+    """Headline size, in the launch configuration the benchmark times.  The
+    oracle routes the full permutation once (about two minutes on one core)."""
+    n = 26
+    perm = inputs.random_perm(n, 2)
+    bits = gpu_route(perm, n)
+    x = inputs.payload_u64(1 << n, 2)
+    out = gpu_apply(bits, x, n)
+    assert np.array_equal(out, x[perm])
+    assert np.array_equal(bits, oracle.route(perm, n))
+
+
+# ---- host-buffer entry points, validation, robustness -------------------------------------------
+def test_host_entry_points():
+    n, batch = 15, 2
+    perm = inputs.random_perm_batch(n, batch, seed0=5)
+    bits = np.empty((batch, 2 * n - 1, (1 << n) // 64), dtype=np.uint32)
+    binding.benes_route_host(perm, n, batch, bits)
+    assert np.array_equal(bits, oracle.route(perm, n))
+    x = inputs.payload_u64(batch << n, 4).reshape(batch, -1)
+    out = np.empty_like(x)
+    binding.benes_apply_host(bits, x, out, 8, n, batch)
+    assert np.array_equal(out, np.take_along_axis(x, perm.astype(np.int64), axis=1))
+
+
+def test_caller_workspace_is_used_and_checked():
+    n = 15
+    perm = inputs.random_perm(n, 11)
+    need = binding.benes_route_workspace_bytes(n, 1)
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    try:
+        binding.benes_set_workspace(ws)
+        assert np.array_equal(gpu_route(perm, n), oracle.route(perm, n))
+        binding.benes_set_workspace(ws, 4096)       # too small for this call
+        with pytest.raises(binding.BenesError) as e:
+            gpu_route(perm, n)
+        assert e.value.status == binding.BENES_ERR_NOMEM
+    finally:
+        binding.benes_set_workspace(None)
+
+
+@pytest.mark.parametrize("n,batch", [(3, 4), (8, 10), (14, 2)])
+def test_validate_perm(n, batch):
+    perm = inputs.random_perm_batch(n, batch, seed0=1)
+    assert binding.benes_validate_perm(dev(perm), n, batch)
+    bad = perm.copy()
+    bad[batch - 1, 3] = bad[batch - 1, 4]           # a duplicate
+    assert not binding.benes_validate_perm(dev(bad), n, batch)
+    bad = perm.copy()
+    bad[0, 0] = 1 << n                              # out of range
+    assert not binding.benes_validate_perm(dev(bad), n, batch)
+
+
+@pytest.mark.parametrize("n", [6, 14])
+def test_non_permutation_input_is_memory_safe(n):
+    """Every index the kernels form is masked to its block, so duplicated values
+    give an unspecified setting but no error; a good call afterwards is exact."""
+    bad = inputs.random_perm(n, 2)
+    bad[1::2] = bad[0::2]
+    gpu_route(bad, n)
+    assert torch.cuda.current_stream().query() or True
+    torch.cuda.synchronize()
+    perm = inputs.random_perm(n, 3)
+    assert np.array_equal(gpu_route(perm, n), oracle.route(perm, n))
+
+
+def test_launch_counter_counts():
+    n = 14
+    before = binding.benes_launch_count()
+    gpu_route(inputs.random_perm(n, 1), n)
+    after = binding.benes_launch_count()
+    assert after > before
