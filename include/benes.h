@@ -120,6 +120,21 @@ int benes_validate_perm(const uint32_t *perm, int log2n, int batch, benes_stream
 /* Kernels launched by this library in this process so far (host-side counter). */
 unsigned long long benes_launch_count(void);
 
+/*
+ * Optional per-kernel timing.  While enabled, the library brackets each group
+ * of consecutive launches of one kernel kind with a pair of CUDA events on the
+ * caller's stream.  benes_profile_read synchronises those events and returns,
+ * for one kind, the launches and the summed device time since the last reset.
+ * Kinds: 0 inverse scatter, 1 successor build, 2 pointer-jumping pass,
+ * 3 last pass + output-side bits, 4 input-side bits + compaction, 5 fused
+ * in-CTA levels, 6 payload-apply stage.  BENES_PROFILE_KINDS = number of kinds.
+ */
+#define BENES_PROFILE_KINDS 7
+int benes_profile_enable(int on);
+int benes_profile_reset(void);
+int benes_profile_read(int kind, unsigned long long *launches, double *milliseconds);
+const char *benes_profile_kind_name(int kind);
+
 /* Largest block size (log2) finished inside one CTA by the fused kernel. */
 int benes_fused_log2m(void);
 

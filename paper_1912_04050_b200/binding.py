@@ -37,6 +37,10 @@ SYMBOLS = {
     "benes_release_workspace": (_i, []),
     "benes_validate_perm": (_i, [_vp, _i, _i, _vp]),
     "benes_launch_count": (ctypes.c_ulonglong, []),
+    "benes_profile_enable": (_i, [_i]),
+    "benes_profile_reset": (_i, []),
+    "benes_profile_read": (_i, [_i, ctypes.POINTER(ctypes.c_ulonglong), ctypes.POINTER(ctypes.c_double)]),
+    "benes_profile_kind_name": (ctypes.c_char_p, [_i]),
     "benes_fused_log2m": (_i, []),
     "benes_status_string": (ctypes.c_char_p, [_i]),
 }
@@ -162,6 +166,28 @@ def benes_validate_perm(perm: torch.Tensor, log2n: int, batch: int, stream=None)
 
 def benes_launch_count() -> int:
     return load().benes_launch_count()
+
+
+PROFILE_KINDS = 7
+
+
+def benes_profile_enable(on: bool) -> None:
+    _check(load().benes_profile_enable(1 if on else 0), "benes_profile_enable")
+
+
+def benes_profile_reset() -> None:
+    _check(load().benes_profile_reset(), "benes_profile_reset")
+
+
+def benes_profile_read(kind: int):
+    """(launches, milliseconds) of one kernel kind since the last reset."""
+    n, ms = ctypes.c_ulonglong(0), ctypes.c_double(0.0)
+    _check(load().benes_profile_read(kind, ctypes.byref(n), ctypes.byref(ms)), "benes_profile_read")
+    return n.value, ms.value
+
+
+def benes_profile_kind_name(kind: int) -> str:
+    return load().benes_profile_kind_name(kind).decode()
 
 
 def benes_fused_log2m() -> int:

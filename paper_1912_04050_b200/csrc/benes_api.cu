@@ -93,21 +93,37 @@ int route_levels(const uint32_t *perm, int n, size_t batch, uint32_t *bits, char
     BitsLayout L{bits, n, n - 6};
     const uint32_t *P = perm;
     uint32_t *Q = Qbuf[0];
-    int rc = launch_inverse(P, Q, T, n, s);
-    if (rc) return rc;
+    int rc;
+    {
+        ProfileScope ps(kInverse, s);
+        if ((rc = launch_inverse(P, Q, T, n, s))) return rc;
+    }
     int cur = 0;
     for (int level = 0; n - level > kFusedLog2M; ++level) {
         const int m = n - level;
-        if ((rc = launch_build(P, Q, Wd, T, m, s))) return rc;
-        for (int r = 1; r < m - 1; ++r)
-            if ((rc = launch_jump(Wd, T, s))) return rc;
-        if ((rc = launch_jump_last(Wd, T, L, 2 * n - 2 - level, s))) return rc;
+        {
+            ProfileScope ps(kBuild, s);
+            if ((rc = launch_build(P, Q, Wd, T, m, s))) return rc;
+        }
+        {
+            ProfileScope ps(kJump, s);
+            for (int r = 1; r < m - 1; ++r)
+                if ((rc = launch_jump(Wd, T, s))) return rc;
+        }
+        {
+            ProfileScope ps(kJumpLast, s);
+            if ((rc = launch_jump_last(Wd, T, L, 2 * n - 2 - level, s))) return rc;
+        }
         uint32_t *Pn = Pbuf[cur], *Qn = Qbuf[cur ^ 1];
-        if ((rc = launch_split(P, Q, Pn, Qn, T, m, L, level, 2 * n - 2 - level, s))) return rc;
+        {
+            ProfileScope ps(kSplit, s);
+            if ((rc = launch_split(P, Q, Pn, Qn, T, m, L, level, 2 * n - 2 - level, s))) return rc;
+        }
         P = Pn;
         Q = Qn;
         cur ^= 1;
     }
+    ProfileScope ps(kFused, s);
     return launch_fused(P, T, kFusedLog2M, bits, n, s);
 }
 
@@ -168,6 +184,7 @@ int benes_route(const uint32_t *perm, int log2n, int batch, uint32_t *switch_bit
     if (n <= kFusedLog2M) {
         // whole permutations fit one CTA each
         const size_t max_ctas = size_t(1) << 30;
+        ProfileScope ps(kFused, s);
         for (size_t b0 = 0; b0 < size_t(batch); b0 += max_ctas) {
             size_t nb = size_t(batch) - b0 < max_ctas ? size_t(batch) - b0 : max_ctas;
             int rc = launch_fused(perm + (b0 << n), nb << n, n,
@@ -204,6 +221,7 @@ int benes_apply_ex(const uint32_t *switch_bits, const void *in, void *out, int e
     }
     // ping-pong between `out` and the scratch buffer so that the last stage lands in `out`
     const void *src = in;
+    ProfileScope ps(kApply, s);
     for (int st = 0; st < stages; ++st) {
         void *dst = ((stages - 1 - st) % 2 == 0) ? out : ws;
         int rc = launch_apply_stage(switch_bits, src, dst, elem_bytes, st, n, size_t(batch), s);

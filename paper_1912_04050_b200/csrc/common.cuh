@@ -27,6 +27,17 @@ inline int launch_status() {
     return cudaPeekAtLastError() == cudaSuccess ? BENES_OK : BENES_ERR_CUDA;
 }
 
+// Optional event timing of a group of launches of one kind (see benes.h).
+enum ProfileKind { kInverse = 0, kBuild, kJump, kJumpLast, kSplit, kFused, kApply };
+struct ProfileScope {
+    ProfileScope(int kind, cudaStream_t s);
+    ~ProfileScope();
+    int kind_;
+    cudaStream_t s_;
+    int slot_;
+    unsigned long long launches0_;
+};
+
 // Where the words of one stage live.  T = flat switch-word index over the
 // whole batch (flat switch index >> 5); valid when N >= 64, so that a word
 // never straddles two permutations.
