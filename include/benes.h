@@ -52,7 +52,8 @@ enum {
     BENES_ERR_BADARG = -1,          /* null pointer, log2n or batch out of range, bad elem_bytes */
     BENES_ERR_CUDA = -2,            /* a CUDA runtime call or launch failed */
     BENES_ERR_NOMEM = -3,           /* workspace could not be allocated / supplied one too small */
-    BENES_ERR_NOT_PERMUTATION = -4  /* benes_validate_perm only */
+    BENES_ERR_NOT_PERMUTATION = -4, /* benes_validate_perm only */
+    BENES_ERR_TOO_LARGE = -5        /* benes_apply_static only: payload exceeds the built-in scratch */
 };
 
 #define BENES_MAX_LOG2N 30
@@ -82,6 +83,33 @@ int benes_apply(const uint32_t *switch_bits, const void *in, void *out, int log2
 /* Same with an explicit element size: elem_bytes must be 4 or 8. */
 int benes_apply_ex(const uint32_t *switch_bits, const void *in, void *out, int elem_bytes,
                    int log2n, int batch, benes_stream_t stream);
+
+/*
+ * benes_apply_ex for callers that cannot allocate device memory.  (The paper
+ * has no counterpart; this is a deployment convenience of this library.)
+ *
+ * Who needs it: a process that has given all device memory to another
+ * allocator, where the cudaMalloc behind the library workspace would fail, and
+ * a latency-critical loop that cannot take the device-wide stall of a
+ * cudaMalloc / cudaFree.  This entry point never calls cudaMalloc, cudaFree or
+ * any allocating routine: its one scratch buffer is a fixed array of
+ * BENES_STATIC_SCRATCH_BYTES that is part of the library image (every GPU
+ * that loads the library keeps it until the process exits).
+ *
+ * Same arguments, layout and result as benes_apply_ex, with one limit:
+ * batch * N * elem_bytes must not exceed BENES_STATIC_SCRATCH_BYTES, otherwise
+ * BENES_ERR_TOO_LARGE is returned and nothing is enqueued.
+ *
+ * The first call on each device looks up the array's device address (a
+ * runtime query, no allocation); make that first call outside any stream
+ * capture.  All calls share the one array and it keeps the previous call's
+ * contents (nothing needs clearing: each stage overwrites all it later
+ * reads).  Two calls whose kernels can overlap on the GPU (different streams,
+ * no ordering) race on it: keep them on one stream or order them yourself.
+ */
+#define BENES_STATIC_SCRATCH_BYTES (4u << 20)
+int benes_apply_static(const uint32_t *switch_bits, const void *in, void *out, int elem_bytes,
+                       int log2n, int batch, benes_stream_t stream);
 
 /*
  * Host-buffer variants: copy the inputs to the device, run, copy the result

@@ -21,6 +21,8 @@ BENES_ERR_BADARG = -1
 BENES_ERR_CUDA = -2
 BENES_ERR_NOMEM = -3
 BENES_ERR_NOT_PERMUTATION = -4
+BENES_ERR_TOO_LARGE = -5
+STATIC_SCRATCH_BYTES = 4 << 20
 
 # every symbol include/benes.h declares: name -> (restype, argtypes)
 _vp, _i, _sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
@@ -28,6 +30,7 @@ SYMBOLS = {
     "benes_route": (_i, [_vp, _i, _i, _vp, _vp]),
     "benes_apply": (_i, [_vp, _vp, _vp, _i, _i, _vp]),
     "benes_apply_ex": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp]),
+    "benes_apply_static": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp]),
     "benes_route_host": (_i, [_vp, _i, _i, _vp, _vp]),
     "benes_apply_host": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp]),
     "benes_switch_words": (_sz, [_i, _i]),
@@ -127,6 +130,15 @@ def benes_apply_ex(switch_bits: torch.Tensor, inp: torch.Tensor, out: torch.Tens
     _check(load().benes_apply_ex(_dev_ptr(switch_bits, "switch_bits"), _dev_ptr(inp, "in"),
                                  _dev_ptr(out, "out"), elem_bytes, log2n, batch, _stream(stream)),
            "benes_apply_ex")
+
+
+def benes_apply_static(switch_bits: torch.Tensor, inp: torch.Tensor, out: torch.Tensor, elem_bytes: int,
+                       log2n: int, batch: int, stream=None) -> None:
+    """benes_apply_ex without any allocation: the scratch is a fixed 4 MiB array inside the
+    library, so batch * N * elem_bytes must fit in it (BenesError with BENES_ERR_TOO_LARGE if not)."""
+    _check(load().benes_apply_static(_dev_ptr(switch_bits, "switch_bits"), _dev_ptr(inp, "in"),
+                                     _dev_ptr(out, "out"), elem_bytes, log2n, batch, _stream(stream)),
+           "benes_apply_static")
 
 
 def benes_route_host(perm_host, log2n: int, batch: int, switch_bits_host, stream=None) -> None:

@@ -310,6 +310,7 @@ const char *benes_status_string(int status) {
         case BENES_ERR_CUDA: return "CUDA runtime error";
         case BENES_ERR_NOMEM: return "workspace allocation failed or caller workspace too small";
         case BENES_ERR_NOT_PERMUTATION: return "input is not a permutation";
+        case BENES_ERR_TOO_LARGE: return "payload larger than the built-in scratch of benes_apply_static";
         default: return "unknown status";
     }
 }
