@@ -37,12 +37,26 @@ WORKLOADS = {
     "c5s": (24, 1, 4, 3, "C5: 1 x N=2^24 Sattolo single-cycle permutation (seed 3), route + uint32 payload apply"),
 }
 
-# Algorithmic bytes of one pointer-jumping pass per element: own 64-bit word read,
-# one 64-bit word gathered, own word written back.
-JUMP_BYTES_PER_ELEMENT = 24.0
-# DRAM bytes per pointer-jumping launch per element measured with ncu
-# (dram__bytes_read.sum + dram__bytes_write.sum); see profiles/.  None until captured.
-JUMP_NCU_DRAM_BYTES_PER_ELEMENT = None
+def algorithmic_bytes_per_element(kind: str, ebytes: int, kappa: int) -> float:
+    """Useful bytes one launch of a kernel kind moves per permutation element."""
+    return {
+        # own 64-bit word read, one 64-bit word gathered, own word written back
+        "jump": 24.0,
+        # per output on a walk: P[j^1] and Q[.] gathered (4 B each), the owner stamp
+        # of its switch (4 B per 2 outputs), one contracted word per 2^kappa outputs
+        "walk": 8.0 + 2.0 + 8.0 / (1 << max(kappa, 1)),
+        # payload pair in, pair out, one switch bit per pair
+        "apply": 2.0 * ebytes + 1.0 / 16.0,
+        "inverse": 8.0, "build": 16.0, "split": 16.25, "colour": 2.0 + 4.0 + 1.0 / 16.0,
+        "jump_last": 8.0 + 1.0 / 16.0, "ruler_jump": 24.0 / (1 << max(kappa, 1)),
+        "fused": 4.0 + (2 * 13 - 1) / 16.0,
+    }[kind]
+
+
+# DRAM bytes per launch per element of the dominant kernel measured with ncu
+# (dram__bytes_read.sum + dram__bytes_write.sum); see profiles/.  None until captured
+# for the kernel as it stands.
+NCU_DRAM_BYTES_PER_ELEMENT = {}
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -228,6 +242,8 @@ def run_gpu(args):
     if dist:
         dist.barrier()
     binding.load()
+    if args.kappa is not None:
+        binding.benes_set_option(binding.OPT_SAMPLE_LOG2K, args.kappa)
 
     name = args.workload
     n, batch, ebytes, seed, desc = WORKLOADS[name]
@@ -326,19 +342,22 @@ def run_gpu(args):
 
     if rank == 0:
         peak, peak_kind = measured_peaks()
-        jump = kinds["jump"]
+        kappa = binding.benes_get_option(binding.OPT_SAMPLE_LOG2K)
+        top = max(kinds, key=lambda k: kinds[k]["ms"])
+        dom = kinds[top]
         roofline = None
-        if jump["launches"]:
-            per_launch_s = jump["ms"] * 1e-3 / jump["launches"]
-            achieved = JUMP_BYTES_PER_ELEMENT * elems / per_launch_s / 1e9
+        if dom["launches"]:
+            per_launch_s = dom["ms"] * 1e-3 / dom["launches"]
+            bpe = algorithmic_bytes_per_element(top, ebytes, kappa)
+            achieved = bpe * elems / per_launch_s / 1e9
             roofline = {
-                "bound": "hbm", "kernel": "k_jump (pointer-jumping pass)",
+                "bound": "hbm", "kernel": top,
                 "achieved": achieved, "peak": peak, "peak_source": peak_kind + " (STREAM-style copy)",
                 "unit": "GB/s", "frac": achieved / peak,
-                "traffic": (JUMP_NCU_DRAM_BYTES_PER_ELEMENT * elems
-                            if JUMP_NCU_DRAM_BYTES_PER_ELEMENT else None),
-                "algorithmic_bytes_per_launch": JUMP_BYTES_PER_ELEMENT * elems,
-                "avg_launch_ms": per_launch_s * 1e3, "launches_timed": jump["launches"],
+                "traffic": (NCU_DRAM_BYTES_PER_ELEMENT[top] * elems
+                            if top in NCU_DRAM_BYTES_PER_ELEMENT else None),
+                "algorithmic_bytes_per_launch": bpe * elems,
+                "avg_launch_ms": per_launch_s * 1e3, "launches_timed": dom["launches"],
             }
         bits_bytes = d_bits.numel() * 4
         line = {
@@ -349,7 +368,8 @@ def run_gpu(args):
             "config": {"workload": desc, "log2n": n, "batch_per_gpu": batch, "payload_bytes": ebytes,
                        "parallelism": "replicas x%d, no collective" % world,
                        "l2": "inputs larger than L2 (perm %d MiB, words %d MiB)" % (elems * 4 >> 20, elems * 8 >> 20),
-                       "fused_log2m": binding.benes_fused_log2m()},
+                       "fused_log2m": binding.benes_fused_log2m(),
+                       "ruler_spacing_log2": kappa},
             "clocks": clocks,
             "e2e": {"value": world * elems / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
                     "h2d_bytes_per_step": perm_h.nbytes + bits_bytes + x_h.nbytes,
@@ -378,6 +398,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c4", choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--kappa", type=int, default=None,
+                    help="ruler spacing (log2) of the loop labelling; 0 = full pointer jumping")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -145,6 +145,22 @@ int benes_release_workspace(void);
  */
 int benes_validate_perm(const uint32_t *perm, int log2n, int batch, benes_stream_t stream);
 
+/*
+ * Tuning of the loop labelling of benes_route (process-wide; set between calls).
+ *   BENES_OPT_SAMPLE_LOG2K : 0 = label every loop by pointer jumping over all
+ *       outputs; kappa in 2..8 (default 4) = label only one sampled "ruler"
+ *       switch per 2^kappa switches by pointer jumping and reach the rest by
+ *       sequential walks between rulers.  The result is identical either way.
+ *   BENES_OPT_WALK_CAP : hops (1 .. 2^24, default 2^14) after which a walk gives
+ *       up; a level in which that happens is relabelled by full pointer jumping.
+ * benes_set_option returns BENES_OK or BENES_ERR_BADARG; benes_get_option
+ * returns the value, or BENES_ERR_BADARG for an unknown key.
+ */
+#define BENES_OPT_SAMPLE_LOG2K 0
+#define BENES_OPT_WALK_CAP 1
+int benes_set_option(int key, int value);
+int benes_get_option(int key);
+
 /* Kernels launched by this library in this process so far (host-side counter). */
 unsigned long long benes_launch_count(void);
 
@@ -155,9 +171,11 @@ unsigned long long benes_launch_count(void);
  * for one kind, the launches and the summed device time since the last reset.
  * Kinds: 0 inverse scatter, 1 successor build, 2 pointer-jumping pass,
  * 3 last pass + output-side bits, 4 input-side bits + compaction, 5 fused
- * in-CTA levels, 6 payload-apply stage.  BENES_PROFILE_KINDS = number of kinds.
+ * in-CTA levels, 6 payload-apply stage, 7 ruler walk, 8 pointer-jumping pass
+ * over the rulers, 9 colouring from owners + output-side bits.
+ * BENES_PROFILE_KINDS = number of kinds.
  */
-#define BENES_PROFILE_KINDS 7
+#define BENES_PROFILE_KINDS 10
 int benes_profile_enable(int on);
 int benes_profile_reset(void);
 int benes_profile_read(int kind, unsigned long long *launches, double *milliseconds);

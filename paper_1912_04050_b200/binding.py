@@ -39,6 +39,8 @@ SYMBOLS = {
     "benes_set_workspace": (_i, [_vp, _sz]),
     "benes_release_workspace": (_i, []),
     "benes_validate_perm": (_i, [_vp, _i, _i, _vp]),
+    "benes_set_option": (_i, [_i, _i]),
+    "benes_get_option": (_i, [_i]),
     "benes_launch_count": (ctypes.c_ulonglong, []),
     "benes_profile_enable": (_i, [_i]),
     "benes_profile_reset": (_i, []),
@@ -180,7 +182,20 @@ def benes_launch_count() -> int:
     return load().benes_launch_count()
 
 
-PROFILE_KINDS = 7
+PROFILE_KINDS = 10
+OPT_SAMPLE_LOG2K = 0
+OPT_WALK_CAP = 1
+
+
+def benes_set_option(key: int, value: int) -> None:
+    _check(load().benes_set_option(key, value), "benes_set_option")
+
+
+def benes_get_option(key: int) -> int:
+    v = load().benes_get_option(key)
+    if v < 0:
+        _check(v, "benes_get_option")
+    return v
 
 
 def benes_profile_enable(on: bool) -> None:

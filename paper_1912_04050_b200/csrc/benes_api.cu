@@ -22,6 +22,12 @@ struct Workspace {
 Workspace g_ws[kMaxDevices];
 std::mutex g_mu;
 
+// Tuning (benes_set_option).  kappa = 0: every loop is labelled by pointer
+// jumping over all outputs; 2..8: one ruler switch per 2^kappa switches.
+int g_kappa = 4;
+int g_walk_cap = 1 << 14;
+constexpr int kMaxLevels = 32;
+
 inline size_t align_up(size_t v) { return (v + kAlign - 1) & ~(kAlign - 1); }
 
 // Returns a device scratch buffer of at least `bytes`.
@@ -70,8 +76,10 @@ inline size_t level_chunk(int log2n, size_t batch) {
 size_t route_ws_bytes(int log2n, size_t batch) {
     if (log2n <= kFusedLog2M) return 0;
     size_t T = level_chunk(log2n, batch) << log2n;
-    // Pa, Pb, Qa, Qb (uint32) + words (uint64)
-    return 4 * align_up(T * 4) + align_up(T * 8);
+    // Pa, Pb, Qa, Qb (uint32) + words (uint64) + owners (uint32 per switch)
+    // + contracted words (at most T/4) + per-level gate flags
+    return 4 * align_up(T * 4) + align_up(T * 8) + align_up(T * 2) + align_up(T * 2) +
+           align_up(kMaxLevels * 4);
 }
 
 size_t apply_ws_bytes(int elem_bytes, int log2n, size_t batch) {
@@ -88,7 +96,13 @@ int route_levels(const uint32_t *perm, int n, size_t batch, uint32_t *bits, char
     Pbuf[1] = reinterpret_cast<uint32_t *>(ws + off); off += align_up(T * 4);
     Qbuf[0] = reinterpret_cast<uint32_t *>(ws + off); off += align_up(T * 4);
     Qbuf[1] = reinterpret_cast<uint32_t *>(ws + off); off += align_up(T * 4);
-    unsigned long long *Wd = reinterpret_cast<unsigned long long *>(ws + off);
+    unsigned long long *Wd = reinterpret_cast<unsigned long long *>(ws + off); off += align_up(T * 8);
+    uint32_t *owner = reinterpret_cast<uint32_t *>(ws + off); off += align_up(T * 2);
+    unsigned long long *Wc = reinterpret_cast<unsigned long long *>(ws + off); off += align_up(T * 2);
+    uint32_t *gates = reinterpret_cast<uint32_t *>(ws + off);
+    const int kappa = g_kappa;
+    const uint32_t cap = uint32_t(g_walk_cap);
+    if (kappa) BENES_CUDA_TRY(cudaMemsetAsync(gates, 0, kMaxLevels * 4, s));
 
     BitsLayout L{bits, n, n - 6};
     const uint32_t *P = perm;
@@ -101,18 +115,41 @@ int route_levels(const uint32_t *perm, int n, size_t batch, uint32_t *bits, char
     int cur = 0;
     for (int level = 0; n - level > kFusedLog2M; ++level) {
         const int m = n - level;
+        const int out_stage = 2 * n - 2 - level;
+        uint32_t *gate = nullptr;
+        if (kappa) {
+            // ruler-sampled labelling; raises `gate` if a walk had to give up
+            gate = gates + level;
+            BENES_CUDA_TRY(cudaMemsetAsync(owner, 0xFF, T * 2, s));
+            {
+                ProfileScope ps(kWalk, s);
+                if ((rc = launch_walk(P, Q, owner, Wc, T, m, kappa, uint32_t(level), cap, gate, s)))
+                    return rc;
+            }
+            {
+                ProfileScope ps(kRulerJump, s);
+                for (int r = 0; r < m - 1 - kappa; ++r)
+                    if ((rc = launch_jump(Wc, T >> kappa, nullptr, s))) return rc;
+            }
+            {
+                ProfileScope ps(kColour, s);
+                if ((rc = launch_colour(P, Q, owner, Wc, T, m, L, out_stage, cap, gate, s))) return rc;
+            }
+        }
+        // pointer jumping over all outputs: the whole labelling when sampling is
+        // off, otherwise gated (a no-op unless this level's walks gave up)
         {
             ProfileScope ps(kBuild, s);
-            if ((rc = launch_build(P, Q, Wd, T, m, s))) return rc;
+            if ((rc = launch_build(P, Q, Wd, T, m, gate, s))) return rc;
         }
         {
             ProfileScope ps(kJump, s);
             for (int r = 1; r < m - 1; ++r)
-                if ((rc = launch_jump(Wd, T, s))) return rc;
+                if ((rc = launch_jump(Wd, T, gate, s))) return rc;
         }
         {
             ProfileScope ps(kJumpLast, s);
-            if ((rc = launch_jump_last(Wd, T, L, 2 * n - 2 - level, s))) return rc;
+            if ((rc = launch_jump_last(Wd, T, L, out_stage, gate, s))) return rc;
         }
         uint32_t *Pn = Pbuf[cur], *Qn = Qbuf[cur ^ 1];
         {
@@ -300,6 +337,30 @@ int benes_validate_perm(const uint32_t *perm, int log2n, int batch, benes_stream
 }
 
 unsigned long long benes_launch_count(void) { return g_launches; }
+
+int benes_set_option(int key, int value) {
+    std::lock_guard<std::mutex> lk(g_mu);
+    switch (key) {
+        case BENES_OPT_SAMPLE_LOG2K:
+            if (value != 0 && (value < 2 || value > 8)) return BENES_ERR_BADARG;
+            g_kappa = value;
+            return BENES_OK;
+        case BENES_OPT_WALK_CAP:
+            if (value < 1 || value > (1 << 24)) return BENES_ERR_BADARG;
+            g_walk_cap = value;
+            return BENES_OK;
+        default: return BENES_ERR_BADARG;
+    }
+}
+
+int benes_get_option(int key) {
+    std::lock_guard<std::mutex> lk(g_mu);
+    switch (key) {
+        case BENES_OPT_SAMPLE_LOG2K: return g_kappa;
+        case BENES_OPT_WALK_CAP: return g_walk_cap;
+        default: return BENES_ERR_BADARG;
+    }
+}
 
 int benes_fused_log2m(void) { return kFusedLog2M; }
 

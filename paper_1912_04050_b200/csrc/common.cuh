@@ -28,7 +28,7 @@ inline int launch_status() {
 }
 
 // Optional event timing of a group of launches of one kind (see benes.h).
-enum ProfileKind { kInverse = 0, kBuild, kJump, kJumpLast, kSplit, kFused, kApply };
+enum ProfileKind { kInverse = 0, kBuild, kJump, kJumpLast, kSplit, kFused, kApply, kWalk, kRulerJump, kColour };
 struct ProfileScope {
     ProfileScope(int kind, cudaStream_t s);
     ~ProfileScope();
@@ -55,13 +55,25 @@ struct BitsLayout {
 // ---- per-level HBM path (route_levels.cu) ----------------------------------
 // total = batch * N flat elements (<= 2^31), all blocks of one level per launch.
 int launch_inverse(const uint32_t *P, uint32_t *Q, size_t total, int log2m, cudaStream_t s);
+// `gate` (may be null): device word; the kernel does nothing while it is 0.
 int launch_build(const uint32_t *P, const uint32_t *Q, unsigned long long *Wd, size_t total,
-                 int log2m, cudaStream_t s);
-int launch_jump(unsigned long long *Wd, size_t total, cudaStream_t s);
+                 int log2m, const uint32_t *gate, cudaStream_t s);
+int launch_jump(unsigned long long *Wd, size_t total, const uint32_t *gate, cudaStream_t s);
 int launch_jump_last(const unsigned long long *Wd, size_t total, BitsLayout L, int out_stage,
-                     cudaStream_t s);
+                     const uint32_t *gate, cudaStream_t s);
 int launch_split(const uint32_t *P, const uint32_t *Q, uint32_t *Pn, uint32_t *Qn, size_t total,
                  int log2m, BitsLayout L, int in_stage, int out_stage, cudaStream_t s);
+
+// ---- ruler-sampled loop labelling (route_sampled.cu) --------------------------
+// One ruler switch per group of 2^kappa switches.  owner: total/2 words, preset
+// to 0xFFFFFFFF; Wc: total >> kappa contracted words; gate: raised when a walk
+// exceeds `cap` hops.
+int launch_walk(const uint32_t *P, const uint32_t *Q, uint32_t *owner, unsigned long long *Wc,
+                size_t total, int log2m, int kappa, uint32_t salt, uint32_t cap, uint32_t *gate,
+                cudaStream_t s);
+int launch_colour(const uint32_t *P, const uint32_t *Q, const uint32_t *owner,
+                  const unsigned long long *Wc, size_t total, int log2m, BitsLayout L,
+                  int out_stage, uint32_t cap, uint32_t *gate, cudaStream_t s);
 
 // ---- fused path (route_fused.cu) -------------------------------------------
 // Finishes levels (n - log2m) .. n-1 of every block of size 2^log2m of the flat

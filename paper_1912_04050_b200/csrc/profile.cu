@@ -29,7 +29,8 @@ cudaEvent_t take_event() {
     return e;
 }
 
-const char *kNames[BENES_PROFILE_KINDS] = {"inverse", "build", "jump", "jump_last", "split", "fused", "apply"};
+const char *kNames[BENES_PROFILE_KINDS] = {"inverse", "build", "jump", "jump_last", "split", "fused", "apply",
+                                           "walk", "ruler_jump", "colour"};
 
 }  // namespace
 

@@ -51,7 +51,8 @@ k_inverse(const uint4 *__restrict__ P4, uint32_t *__restrict__ Q, size_t quads, 
 // Two output switches (four outputs) per thread.
 __global__ void __launch_bounds__(kThreads)
 k_build(const uint4 *__restrict__ P4, const uint32_t *__restrict__ Q,
-        ulonglong2 *__restrict__ W2, size_t quads, uint32_t mmask) {
+        ulonglong2 *__restrict__ W2, size_t quads, uint32_t mmask, const uint32_t *__restrict__ gate) {
+    if (gate && *gate == 0u) return;
     size_t stride = size_t(gridDim.x) * blockDim.x;
     for (size_t i = size_t(blockIdx.x) * blockDim.x + threadIdx.x; i < quads; i += stride) {
         uint4 p = __ldg(P4 + i);
@@ -82,7 +83,8 @@ __device__ __forceinline__ unsigned long long jump(unsigned long long w, unsigne
 // a3: one in-place pointer-jumping pass.  Four words per thread: two 16-byte
 // loads of the thread's own words, four independent 8-byte gathers.
 __global__ void __launch_bounds__(kThreads)
-k_jump(unsigned long long *__restrict__ Wd, size_t quads) {
+k_jump(unsigned long long *__restrict__ Wd, size_t quads, const uint32_t *__restrict__ gate) {
+    if (gate && *gate == 0u) return;
     size_t stride = size_t(gridDim.x) * blockDim.x;
     ulonglong2 *W2 = reinterpret_cast<ulonglong2 *>(Wd);
     for (size_t i = size_t(blockIdx.x) * blockDim.x + threadIdx.x; i < quads; i += stride) {
@@ -104,7 +106,9 @@ k_jump(unsigned long long *__restrict__ Wd, size_t quads) {
 // a3 (last pass) + a4 + out-side half of a5: only the even outputs are
 // needed; colour = leader & 1 goes straight into the output-side stage word.
 __global__ void __launch_bounds__(kThreads)
-k_jump_last(const unsigned long long *__restrict__ Wd, size_t switches, BitsLayout L, int out_stage) {
+k_jump_last(const unsigned long long *__restrict__ Wd, size_t switches, BitsLayout L, int out_stage,
+            const uint32_t *__restrict__ gate) {
+    if (gate && *gate == 0u) return;
     size_t stride = size_t(gridDim.x) * blockDim.x;
     for (size_t t = size_t(blockIdx.x) * blockDim.x + threadIdx.x; t < switches; t += stride) {
         unsigned long long w = __ldcg(Wd + 2 * t);
@@ -166,24 +170,24 @@ int launch_inverse(const uint32_t *P, uint32_t *Q, size_t total, int log2m, cuda
 }
 
 int launch_build(const uint32_t *P, const uint32_t *Q, unsigned long long *Wd, size_t total,
-                 int log2m, cudaStream_t s) {
+                 int log2m, const uint32_t *gate, cudaStream_t s) {
     size_t quads = total / 4;
     k_build<<<grid_for(quads), kThreads, 0, s>>>(reinterpret_cast<const uint4 *>(P), Q,
                                                  reinterpret_cast<ulonglong2 *>(Wd), quads,
-                                                 (1u << log2m) - 1u);
+                                                 (1u << log2m) - 1u, gate);
     return launch_status();
 }
 
-int launch_jump(unsigned long long *Wd, size_t total, cudaStream_t s) {
+int launch_jump(unsigned long long *Wd, size_t total, const uint32_t *gate, cudaStream_t s) {
     size_t quads = total / 4;
-    k_jump<<<grid_for(quads), kThreads, 0, s>>>(Wd, quads);
+    k_jump<<<grid_for(quads), kThreads, 0, s>>>(Wd, quads, gate);
     return launch_status();
 }
 
 int launch_jump_last(const unsigned long long *Wd, size_t total, BitsLayout L, int out_stage,
-                     cudaStream_t s) {
+                     const uint32_t *gate, cudaStream_t s) {
     size_t switches = total / 2;
-    k_jump_last<<<grid_for(switches), kThreads, 0, s>>>(Wd, switches, L, out_stage);
+    k_jump_last<<<grid_for(switches), kThreads, 0, s>>>(Wd, switches, L, out_stage, gate);
     return launch_status();
 }
 

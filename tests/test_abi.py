@@ -67,6 +67,21 @@ def test_argument_errors_are_reported_on_the_host(lib):
     assert lib.benes_set_workspace(ctypes.c_void_p(100), 1024) == binding.BENES_ERR_BADARG  # alignment
 
 
+def test_options_are_validated(lib):
+    k0 = lib.benes_get_option(binding.OPT_SAMPLE_LOG2K)
+    c0 = lib.benes_get_option(binding.OPT_WALK_CAP)
+    assert 2 <= k0 <= 8 and c0 >= 1
+    for bad in (1, 9, -1):
+        assert lib.benes_set_option(binding.OPT_SAMPLE_LOG2K, bad) == binding.BENES_ERR_BADARG
+    assert lib.benes_set_option(binding.OPT_WALK_CAP, 0) == binding.BENES_ERR_BADARG
+    assert lib.benes_set_option(99, 1) == binding.BENES_ERR_BADARG
+    assert lib.benes_get_option(99) == binding.BENES_ERR_BADARG
+    assert lib.benes_set_option(binding.OPT_SAMPLE_LOG2K, 0) == binding.BENES_OK
+    assert lib.benes_get_option(binding.OPT_SAMPLE_LOG2K) == 0
+    assert lib.benes_set_option(binding.OPT_SAMPLE_LOG2K, k0) == binding.BENES_OK
+    assert lib.benes_get_option(binding.OPT_SAMPLE_LOG2K) == k0 and lib.benes_get_option(binding.OPT_WALK_CAP) == c0
+
+
 def test_status_strings(lib):
     assert binding.status_string(0) == "ok"
     seen = {binding.status_string(s) for s in (0, -1, -2, -3, -4)}

@@ -75,6 +75,42 @@ def test_route_exhaustive_n8():
     assert np.array_equal(gpu_route(perms, 3), oracle.route(perms, 3))
 
 
+# ---- loop-labelling variants: all must give the oracle's bits -------------------
+@pytest.fixture
+def labelling_options():
+    k0 = binding.benes_get_option(binding.OPT_SAMPLE_LOG2K)
+    c0 = binding.benes_get_option(binding.OPT_WALK_CAP)
+    yield
+    binding.benes_set_option(binding.OPT_SAMPLE_LOG2K, k0)
+    binding.benes_set_option(binding.OPT_WALK_CAP, c0)
+
+
+@pytest.mark.parametrize("kappa", [0, 2, 3, 5, 8])
+def test_route_every_ruler_spacing(kappa, labelling_options):
+    """0 = pointer jumping over all outputs; otherwise one ruler per 2^kappa switches."""
+    binding.benes_set_option(binding.OPT_SAMPLE_LOG2K, kappa)
+    for n in (14, 17):
+        perm = inputs.random_perm(n, 40 + n)
+        assert np.array_equal(gpu_route(perm, n), oracle.route(perm, n))
+    n = 16
+    for kind, perm in inputs.structured_perms(n).items():
+        assert np.array_equal(gpu_route(perm, n), oracle.route(perm, n)), kind
+    perm = inputs.random_perm_batch(15, 3, seed0=9)
+    assert np.array_equal(gpu_route(perm, 15), oracle.route(perm, 15))
+
+
+@pytest.mark.parametrize("cap", [1, 3, 40])
+def test_route_walks_that_give_up_fall_back_to_full_pointer_jumping(cap, labelling_options):
+    """With a tiny hop limit almost every level raises its gate and is relabelled
+    by the full pointer-jumping kernels; the bits must not change."""
+    binding.benes_set_option(binding.OPT_WALK_CAP, cap)
+    for n in (14, 16):
+        for kind, perm in inputs.structured_perms(n).items():
+            assert np.array_equal(gpu_route(perm, n), oracle.route(perm, n)), kind
+        perm = inputs.random_perm(n, 60 + n)
+        assert np.array_equal(gpu_route(perm, n), oracle.route(perm, n))
+
+
 # ---- apply ------------------------------------------------------------------
 @pytest.mark.parametrize("n", [1, 2, 3, 5, 6, 7, 10, 13, 16])
 @pytest.mark.parametrize("dtype", [np.uint32, np.uint64])
