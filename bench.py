@@ -39,16 +39,24 @@ WORKLOADS = {
 
 def algorithmic_bytes_per_element(kind: str, ebytes: int, kappa: int) -> float:
     """Useful bytes one launch of a kernel kind moves per permutation element."""
+    k = float(1 << max(kappa, 1))
     return {
-        # own 64-bit word read, one 64-bit word gathered, own word written back
-        "jump": 24.0,
-        # per output on a walk: P[j^1] and Q[.] gathered (4 B each), the owner stamp
-        # of its switch (4 B per 2 outputs), one contracted word per 2^kappa outputs
-        "walk": 8.0 + 2.0 + 8.0 / (1 << max(kappa, 1)),
+        # per switch, visited once: P[j^1] read (4 B), owner word read and written (8 B),
+        # Q[.] read (4 B) -> 8 B per element; one 16-byte walk record per ruler output
+        "walk": 8.0 + 16.0 / k,
+        # build 16 B + (m-2) passes of 24 B + last 8 B per element, m ~ 20 on average
+        "full_label": 16.0 + 18 * 24.0 + 8.0,
         # payload pair in, pair out, one switch bit per pair
         "apply": 2.0 * ebytes + 1.0 / 16.0,
-        "inverse": 8.0, "build": 16.0, "split": 16.25, "colour": 2.0 + 4.0 + 1.0 / 16.0,
-        "jump_last": 8.0 + 1.0 / 16.0, "ruler_jump": 24.0 / (1 << max(kappa, 1)),
+        "apply_fused": 2.0 * ebytes + 1.0 / 16.0,
+        # P read (4 B), record written (8 B), Q scattered (4 B)
+        "inverse": 16.0,
+        # record (8 B) and Q (4 B) read, record (8 B) and Q' (4 B) written, two stage bits
+        "split": 24.0 + 1.0 / 8.0,
+        # owner word per switch, contracted word per switch, one stage bit
+        "colour": 2.0 + 4.0 + 1.0 / 16.0,
+        "combine": (16.0 + 16.0 + 8.0) / k, "list_walk": 20.0 / k, "list_label": 16.0 / k / 16.0,
+        "list_resolve": 24.0 / k,
         "fused": 4.0 + (2 * 13 - 1) / 16.0,
     }[kind]
 

@@ -169,13 +169,14 @@ unsigned long long benes_launch_count(void);
  * of consecutive launches of one kernel kind with a pair of CUDA events on the
  * caller's stream.  benes_profile_read synchronises those events and returns,
  * for one kind, the launches and the summed device time since the last reset.
- * Kinds: 0 inverse scatter, 1 successor build, 2 pointer-jumping pass,
- * 3 last pass + output-side bits, 4 input-side bits + compaction, 5 fused
- * in-CTA levels, 6 payload-apply stage, 7 ruler walk, 8 pointer-jumping pass
- * over the rulers, 9 colouring from owners + output-side bits.
+ * Kinds: 0 inverse scatter, 1 pointer jumping over all outputs (one launch per
+ * level), 2 input-side bits + compaction, 3 fused in-CTA levels, 4 payload-apply
+ * stage, 5 ruler walk, 6 contracted-list assembly, 7 walk over a contracted
+ * list, 8 in-CTA labelling of a contracted list, 9 labels back to a sampled
+ * list, 10 colouring + output-side bits, 11 payload-apply over several stages.
  * BENES_PROFILE_KINDS = number of kinds.
  */
-#define BENES_PROFILE_KINDS 10
+#define BENES_PROFILE_KINDS 12
 int benes_profile_enable(int on);
 int benes_profile_reset(void);
 int benes_profile_read(int kind, unsigned long long *launches, double *milliseconds);

@@ -182,7 +182,7 @@ def benes_launch_count() -> int:
     return load().benes_launch_count()
 
 
-PROFILE_KINDS = 10
+PROFILE_KINDS = 12
 OPT_SAMPLE_LOG2K = 0
 OPT_WALK_CAP = 1
 

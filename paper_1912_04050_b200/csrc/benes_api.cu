@@ -73,13 +73,15 @@ inline size_t level_chunk(int log2n, size_t batch) {
     return batch < per ? batch : per;
 }
 
+// Scratch of the per-level path for T flat elements: two generations of switch
+// records (16 B per switch) and of inverses, the 64-bit words of the full
+// pointer jumping, the scratch of the sampled labelling, per-level gate flags.
+constexpr int kMaxKappa = 8, kMinKappa = 2;
 size_t route_ws_bytes(int log2n, size_t batch) {
     if (log2n <= kFusedLog2M) return 0;
     size_t T = level_chunk(log2n, batch) << log2n;
-    // Pa, Pb, Qa, Qb (uint32) + words (uint64) + owners (uint32 per switch)
-    // + contracted words (at most T/4) + per-level gate flags
-    return 4 * align_up(T * 4) + align_up(T * 8) + align_up(T * 2) + align_up(T * 2) +
-           align_up(kMaxLevels * 4);
+    return 2 * align_up(T * 8) + 2 * align_up(T * 4) + align_up(T * 8) +
+           align_up(sampled_scratch_bytes(T, kMinKappa)) + align_up(kMaxLevels * 4);
 }
 
 size_t apply_ws_bytes(int elem_bytes, int log2n, size_t batch) {
@@ -90,78 +92,59 @@ size_t apply_ws_bytes(int elem_bytes, int log2n, size_t batch) {
 // Levels 0 .. n-kFusedLog2M-1 in HBM, then the fused tail.
 int route_levels(const uint32_t *perm, int n, size_t batch, uint32_t *bits, char *ws, cudaStream_t s) {
     const size_t T = batch << n;
-    uint32_t *Pbuf[2], *Qbuf[2];
+    uint4 *Sbuf[2];
+    uint32_t *Qbuf[2];
     size_t off = 0;
-    Pbuf[0] = reinterpret_cast<uint32_t *>(ws + off); off += align_up(T * 4);
-    Pbuf[1] = reinterpret_cast<uint32_t *>(ws + off); off += align_up(T * 4);
+    Sbuf[0] = reinterpret_cast<uint4 *>(ws + off); off += align_up(T * 8);
+    Sbuf[1] = reinterpret_cast<uint4 *>(ws + off); off += align_up(T * 8);
     Qbuf[0] = reinterpret_cast<uint32_t *>(ws + off); off += align_up(T * 4);
     Qbuf[1] = reinterpret_cast<uint32_t *>(ws + off); off += align_up(T * 4);
     unsigned long long *Wd = reinterpret_cast<unsigned long long *>(ws + off); off += align_up(T * 8);
-    uint32_t *owner = reinterpret_cast<uint32_t *>(ws + off); off += align_up(T * 2);
-    unsigned long long *Wc = reinterpret_cast<unsigned long long *>(ws + off); off += align_up(T * 2);
+    char *sampled = ws + off; off += align_up(sampled_scratch_bytes(T, kMinKappa));
     uint32_t *gates = reinterpret_cast<uint32_t *>(ws + off);
     const int kappa = g_kappa;
     const uint32_t cap = uint32_t(g_walk_cap);
-    if (kappa) BENES_CUDA_TRY(cudaMemsetAsync(gates, 0, kMaxLevels * 4, s));
+    SampledScratch sc;
+    int rc;
+    if (kappa) {
+        sampled_scratch_carve(sampled, T, kappa, &sc);
+        BENES_CUDA_TRY(cudaMemsetAsync(gates, 0, kMaxLevels * 4, s));
+        if ((rc = sampled_scratch_reset(sc, T, kappa, s))) return rc;
+    }
 
     BitsLayout L{bits, n, n - 6};
-    const uint32_t *P = perm;
-    uint32_t *Q = Qbuf[0];
-    int rc;
     {
         ProfileScope ps(kInverse, s);
-        if ((rc = launch_inverse(P, Q, T, n, s))) return rc;
+        if ((rc = launch_inverse(perm, Sbuf[0], Qbuf[0], T, n, s))) return rc;
     }
     int cur = 0;
     for (int level = 0; n - level > kFusedLog2M; ++level) {
         const int m = n - level;
         const int out_stage = 2 * n - 2 - level;
+        uint4 *S = Sbuf[cur];
+        uint32_t *Q = Qbuf[cur];
         uint32_t *gate = nullptr;
         if (kappa) {
             // ruler-sampled labelling; raises `gate` if a walk had to give up
             gate = gates + level;
-            BENES_CUDA_TRY(cudaMemsetAsync(owner, 0xFF, T * 2, s));
-            {
-                ProfileScope ps(kWalk, s);
-                if ((rc = launch_walk(P, Q, owner, Wc, T, m, kappa, uint32_t(level), cap, gate, s)))
-                    return rc;
-            }
-            {
-                ProfileScope ps(kRulerJump, s);
-                for (int r = 0; r < m - 1 - kappa; ++r)
-                    if ((rc = launch_jump(Wc, T >> kappa, nullptr, s))) return rc;
-            }
-            {
-                ProfileScope ps(kColour, s);
-                if ((rc = launch_colour(P, Q, owner, Wc, T, m, L, out_stage, cap, gate, s))) return rc;
-            }
+            if ((rc = sampled_label(S, Q, sc, T, m, kappa, uint32_t(level), cap, L, out_stage, gate, s)))
+                return rc;
         }
         // pointer jumping over all outputs: the whole labelling when sampling is
-        // off, otherwise gated (a no-op unless this level's walks gave up)
+        // off, otherwise gated (returns at once unless this level's walks gave up)
         {
-            ProfileScope ps(kBuild, s);
-            if ((rc = launch_build(P, Q, Wd, T, m, gate, s))) return rc;
+            ProfileScope ps(kFullLabel, s);
+            if ((rc = launch_full_label(S, Q, Wd, T, m, L, out_stage, gate, s))) return rc;
         }
-        {
-            ProfileScope ps(kJump, s);
-            for (int r = 1; r < m - 1; ++r)
-                if ((rc = launch_jump(Wd, T, gate, s))) return rc;
-        }
-        {
-            ProfileScope ps(kJumpLast, s);
-            if ((rc = launch_jump_last(Wd, T, L, out_stage, gate, s))) return rc;
-        }
-        uint32_t *Pn = Pbuf[cur], *Qn = Qbuf[cur ^ 1];
         {
             ProfileScope ps(kSplit, s);
-            if ((rc = launch_split(P, Q, Pn, Qn, T, m, L, level, 2 * n - 2 - level, s))) return rc;
+            if ((rc = launch_split(S, Q, Sbuf[cur ^ 1], Qbuf[cur ^ 1], T, m, L, level, out_stage, s)))
+                return rc;
         }
-        P = Pn;
-        Q = Qn;
         cur ^= 1;
     }
     ProfileScope ps(kFused, s);
-    return launch_fused(P, T, kFusedLog2M, bits, n, s);
+    return launch_fused(Sbuf[cur], 1, T, kFusedLog2M, bits, n, s);
 }
 
 }  // namespace
@@ -224,7 +207,7 @@ int benes_route(const uint32_t *perm, int log2n, int batch, uint32_t *switch_bit
         ProfileScope ps(kFused, s);
         for (size_t b0 = 0; b0 < size_t(batch); b0 += max_ctas) {
             size_t nb = size_t(batch) - b0 < max_ctas ? size_t(batch) - b0 : max_ctas;
-            int rc = launch_fused(perm + (b0 << n), nb << n, n,
+            int rc = launch_fused(perm + (b0 << n), 0, nb << n, n,
                                   switch_bits + b0 * size_t(2 * n - 1) * stage_words(n), n, s);
             if (rc) return rc;
         }
@@ -342,7 +325,7 @@ int benes_set_option(int key, int value) {
     std::lock_guard<std::mutex> lk(g_mu);
     switch (key) {
         case BENES_OPT_SAMPLE_LOG2K:
-            if (value != 0 && (value < 2 || value > 8)) return BENES_ERR_BADARG;
+            if (value != 0 && (value < kMinKappa || value > kMaxKappa)) return BENES_ERR_BADARG;
             g_kappa = value;
             return BENES_OK;
         case BENES_OPT_WALK_CAP:

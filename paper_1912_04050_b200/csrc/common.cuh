@@ -13,6 +13,13 @@ namespace benes {
 // the per-level HBM kernels.
 constexpr int kFusedLog2M = 13;
 
+// Largest list (log2 of its 64-bit words) that one CTA labels in shared memory.
+constexpr int kListSmemLog2 = 14;
+// Ruler spacing (log2) used when a contracted list is itself sampled.
+constexpr int kListKappa = 4;
+
+constexpr uint32_t kUnowned = 0xFFFFFFFFu;
+
 // Every kernel launch of the library goes through this counter.
 extern unsigned long long g_launches;
 
@@ -28,7 +35,10 @@ inline int launch_status() {
 }
 
 // Optional event timing of a group of launches of one kind (see benes.h).
-enum ProfileKind { kInverse = 0, kBuild, kJump, kJumpLast, kSplit, kFused, kApply, kWalk, kRulerJump, kColour };
+enum ProfileKind {
+    kInverse = 0, kFullLabel, kSplit, kFused, kApply, kWalk, kCombine, kListWalk, kListLabel,
+    kListResolve, kColour, kApplyFused
+};
 struct ProfileScope {
     ProfileScope(int kind, cudaStream_t s);
     ~ProfileScope();
@@ -52,33 +62,57 @@ struct BitsLayout {
     }
 };
 
+// ---- layout of a level in HBM ------------------------------------------------
+// A level of the per-level path keeps its sub-permutations as one 16-byte
+// record per output switch t of the flat array,
+//     S[t] = { P[2t], P[2t+1], owner, 0 },
+// P block-local, and the inverses Q as a plain uint32 array.  `owner` is
+// kUnowned until a walk of the sampled labelling claims the switch; it sits in
+// the record so that claiming costs no memory access of its own (the walker
+// has just fetched the record for P).
+__device__ __forceinline__ uint32_t rec_p(const uint4 *S, uint32_t j) {
+    return reinterpret_cast<const uint32_t *>(S)[(size_t(j >> 1) << 2) | (j & 1u)];
+}
+
+__device__ __forceinline__ unsigned long long make_word(uint32_t nxt, uint32_t mn) {
+    return (static_cast<unsigned long long>(mn) << 32) | nxt;
+}
+
 // ---- per-level HBM path (route_levels.cu) ----------------------------------
-// total = batch * N flat elements (<= 2^31), all blocks of one level per launch.
-int launch_inverse(const uint32_t *P, uint32_t *Q, size_t total, int log2m, cudaStream_t s);
-// `gate` (may be null): device word; the kernel does nothing while it is 0.
-int launch_build(const uint32_t *P, const uint32_t *Q, unsigned long long *Wd, size_t total,
-                 int log2m, const uint32_t *gate, cudaStream_t s);
-int launch_jump(unsigned long long *Wd, size_t total, const uint32_t *gate, cudaStream_t s);
-int launch_jump_last(const unsigned long long *Wd, size_t total, BitsLayout L, int out_stage,
-                     const uint32_t *gate, cudaStream_t s);
-int launch_split(const uint32_t *P, const uint32_t *Q, uint32_t *Pn, uint32_t *Qn, size_t total,
+// total = batch * N flat elements (<= 2^30), all blocks of one level per launch.
+// Level 0: S records from the caller's permutation, and Q[P[j]] = j.
+int launch_inverse(const uint32_t *perm, uint4 *S, uint32_t *Q, size_t total, int log2m,
+                   cudaStream_t s);
+// Pointer jumping over all outputs (successor build, log2m-2 in-place passes,
+// last pass + output-side bits) in ONE cooperative launch; `gate` (may be
+// null) is a device word: the kernel returns at once while it is 0.
+int launch_full_label(const uint4 *S, const uint32_t *Q, unsigned long long *Wd, size_t total,
+                      int log2m, BitsLayout L, int out_stage, const uint32_t *gate, cudaStream_t s);
+// Input-side bits + next level's records (owner reset) and inverses.
+int launch_split(const uint4 *S, const uint32_t *Q, uint4 *Sn, uint32_t *Qn, size_t total,
                  int log2m, BitsLayout L, int in_stage, int out_stage, cudaStream_t s);
 
 // ---- ruler-sampled loop labelling (route_sampled.cu) --------------------------
-// One ruler switch per group of 2^kappa switches.  owner: total/2 words, preset
-// to 0xFFFFFFFF; Wc: total >> kappa contracted words; gate: raised when a walk
-// exceeds `cap` hops.
-int launch_walk(const uint32_t *P, const uint32_t *Q, uint32_t *owner, unsigned long long *Wc,
-                size_t total, int log2m, int kappa, uint32_t salt, uint32_t cap, uint32_t *gate,
-                cudaStream_t s);
-int launch_colour(const uint32_t *P, const uint32_t *Q, const uint32_t *owner,
-                  const unsigned long long *Wc, size_t total, int log2m, BitsLayout L,
-                  int out_stage, uint32_t cap, uint32_t *gate, cudaStream_t s);
+struct SampledScratch {
+    uint4 *rec;                  // total >> kappa walk records
+    unsigned long long *list[5]; // contracted lists: total >> (kappa + 4 i) words
+    uint32_t *owner[5];          // owners of the words of list[i] (all kUnowned between uses)
+};
+size_t sampled_scratch_bytes(size_t total, int kappa);
+void sampled_scratch_carve(char *base, size_t total, int kappa, SampledScratch *out);
+// Labels every loop of the level and writes the output-side stage; raises
+// *gate if some walk exceeded `cap` hops (the level must then be relabelled).
+int sampled_label(uint4 *S, const uint32_t *Q, const SampledScratch &sc, size_t total, int log2m,
+                  int kappa, uint32_t salt, uint32_t cap, BitsLayout L, int out_stage,
+                  uint32_t *gate, cudaStream_t s);
+// owner[0] and owner[1] must be all kUnowned before the first sampled_label.
+int sampled_scratch_reset(const SampledScratch &sc, size_t total, int kappa, cudaStream_t s);
 
 // ---- fused path (route_fused.cu) -------------------------------------------
 // Finishes levels (n - log2m) .. n-1 of every block of size 2^log2m of the flat
-// array P (total elements), one CTA per block.  log2m <= kFusedLog2M.
-int launch_fused(const uint32_t *P, size_t total, int log2m, uint32_t *bits, int log2n,
+// level array (total elements), one CTA per block.  log2m <= kFusedLog2M.
+// P is a plain uint32 array if records == 0, else the 16-byte switch records.
+int launch_fused(const void *P, int records, size_t total, int log2m, uint32_t *bits, int log2n,
                  cudaStream_t s);
 
 // ---- payload apply (apply.cu) ----------------------------------------------

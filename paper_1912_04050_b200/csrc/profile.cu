@@ -29,8 +29,9 @@ cudaEvent_t take_event() {
     return e;
 }
 
-const char *kNames[BENES_PROFILE_KINDS] = {"inverse", "build", "jump", "jump_last", "split", "fused", "apply",
-                                           "walk", "ruler_jump", "colour"};
+const char *kNames[BENES_PROFILE_KINDS] = {"inverse", "full_label", "split", "fused", "apply", "walk",
+                                           "combine", "list_walk", "list_label", "list_resolve",
+                                           "colour", "apply_fused"};
 
 }  // namespace
 

@@ -26,7 +26,7 @@ struct FusedCfg {
 
 template <int LOGM>
 __global__ void __launch_bounds__(FusedCfg<LOGM>::kThreads)
-k_route_fused(const uint32_t *__restrict__ P, uint32_t *__restrict__ bits, int log2n) {
+k_route_fused(const uint32_t *__restrict__ P, int records, uint32_t *__restrict__ bits, int log2n) {
     using C = FusedCfg<LOGM>;
     constexpr int M = C::M;
     constexpr int T = C::kThreads;
@@ -52,7 +52,12 @@ k_route_fused(const uint32_t *__restrict__ P, uint32_t *__restrict__ bits, int l
     const size_t local_first_switch = (flat0 & (N - 1)) >> 1;
     uint32_t *my_bits = bits + perm * size_t(2 * n - 1) * stage_w + (local_first_switch >> 5);
 
-    for (int j = tid; j < M; j += T) Pa[j] = uint16_t(P[flat0 + j] & uint32_t(M - 1));
+    // plain array, or 16-byte switch records {P[2t], P[2t+1], -, -}
+    for (int j = tid; j < M; j += T) {
+        size_t f = flat0 + j;
+        uint32_t v = records ? P[((f >> 1) << 2) | (f & 1)] : P[f];
+        Pa[j] = uint16_t(v & uint32_t(M - 1));
+    }
     __syncthreads();
 
 #pragma unroll 1
@@ -142,7 +147,7 @@ k_route_fused(const uint32_t *__restrict__ P, uint32_t *__restrict__ bits, int l
 }
 
 template <int LOGM>
-int launch_one(const uint32_t *P, size_t total, uint32_t *bits, int log2n, cudaStream_t s) {
+int launch_one(const uint32_t *P, int records, size_t total, uint32_t *bits, int log2n, cudaStream_t s) {
     using C = FusedCfg<LOGM>;
     static bool configured = false;
     if (!configured && C::kSmemBytes > 48 * 1024) {
@@ -152,28 +157,29 @@ int launch_one(const uint32_t *P, size_t total, uint32_t *bits, int log2n, cudaS
         configured = true;
     }
     size_t blocks = total >> LOGM;
-    k_route_fused<LOGM><<<unsigned(blocks), C::kThreads, C::kSmemBytes, s>>>(P, bits, log2n);
+    k_route_fused<LOGM><<<unsigned(blocks), C::kThreads, C::kSmemBytes, s>>>(P, records, bits, log2n);
     return launch_status();
 }
 
 }  // namespace
 
-int launch_fused(const uint32_t *P, size_t total, int log2m, uint32_t *bits, int log2n,
+int launch_fused(const void *Pv, int records, size_t total, int log2m, uint32_t *bits, int log2n,
                  cudaStream_t s) {
+    const uint32_t *P = static_cast<const uint32_t *>(Pv);
     switch (log2m) {
-        case 1: return launch_one<1>(P, total, bits, log2n, s);
-        case 2: return launch_one<2>(P, total, bits, log2n, s);
-        case 3: return launch_one<3>(P, total, bits, log2n, s);
-        case 4: return launch_one<4>(P, total, bits, log2n, s);
-        case 5: return launch_one<5>(P, total, bits, log2n, s);
-        case 6: return launch_one<6>(P, total, bits, log2n, s);
-        case 7: return launch_one<7>(P, total, bits, log2n, s);
-        case 8: return launch_one<8>(P, total, bits, log2n, s);
-        case 9: return launch_one<9>(P, total, bits, log2n, s);
-        case 10: return launch_one<10>(P, total, bits, log2n, s);
-        case 11: return launch_one<11>(P, total, bits, log2n, s);
-        case 12: return launch_one<12>(P, total, bits, log2n, s);
-        case 13: return launch_one<13>(P, total, bits, log2n, s);
+        case 1: return launch_one<1>(P, records, total, bits, log2n, s);
+        case 2: return launch_one<2>(P, records, total, bits, log2n, s);
+        case 3: return launch_one<3>(P, records, total, bits, log2n, s);
+        case 4: return launch_one<4>(P, records, total, bits, log2n, s);
+        case 5: return launch_one<5>(P, records, total, bits, log2n, s);
+        case 6: return launch_one<6>(P, records, total, bits, log2n, s);
+        case 7: return launch_one<7>(P, records, total, bits, log2n, s);
+        case 8: return launch_one<8>(P, records, total, bits, log2n, s);
+        case 9: return launch_one<9>(P, records, total, bits, log2n, s);
+        case 10: return launch_one<10>(P, records, total, bits, log2n, s);
+        case 11: return launch_one<11>(P, records, total, bits, log2n, s);
+        case 12: return launch_one<12>(P, records, total, bits, log2n, s);
+        case 13: return launch_one<13>(P, records, total, bits, log2n, s);
         default: return BENES_ERR_BADARG;
     }
 }

@@ -2,7 +2,12 @@
 // fit one CTA's shared memory.  One launch covers all 2^l blocks of a level
 // (and all permutations of a batch): arrays are flat, a block of size
 // M = 2^log2m owns flat indices [bM, (b+1)M), and P / Q hold block-local
-// values.
+// values.  P lives in 16-byte switch records (see common.cuh).
+//
+// This file: the level-0 inverse scatter, the compaction that forms the next
+// level, and pointer jumping over ALL outputs (one cooperative kernel), which
+// is the labelling when sampling is switched off and the fallback when a walk
+// of the sampled labelling gives up.
 //
 // Words of the pointer-jumping array: one 64-bit word per output,
 //   low 32 bits  = nxt (flat index of the current successor),
@@ -11,6 +16,10 @@
 // the in-place update safe: whenever a word is read it satisfies
 // "mn = min over the g-path from j up to, but excluding, nxt".
 #include "common.cuh"
+
+#include <cooperative_groups.h>
+
+namespace cg = cooperative_groups;
 
 namespace benes {
 
@@ -27,50 +36,24 @@ inline int grid_for(size_t work_items, int per_sm = 8) {
     return int(blocks < cap ? (blocks ? blocks : 1) : cap);
 }
 
-__device__ __forceinline__ unsigned long long make_word(uint32_t nxt, uint32_t mn) {
-    return (static_cast<unsigned long long>(mn) << 32) | nxt;
-}
-
-// a1: Q[base + P[j]] = j - base.  Four elements per thread, 16-byte loads.
+// a1 at level 0: records of two switches per thread (16-byte load of four
+// values of the caller's permutation) and Q[base + P[j]] = j - base.
 __global__ void __launch_bounds__(kThreads)
-k_inverse(const uint4 *__restrict__ P4, uint32_t *__restrict__ Q, size_t quads, uint32_t mmask) {
+k_inverse(const uint4 *__restrict__ P4, uint4 *__restrict__ S, uint32_t *__restrict__ Q,
+          size_t quads, uint32_t mmask) {
     size_t stride = size_t(gridDim.x) * blockDim.x;
     for (size_t i = size_t(blockIdx.x) * blockDim.x + threadIdx.x; i < quads; i += stride) {
-        uint4 p = __ldg(P4 + i);
+        uint4 p = __ldcs(P4 + i);
+        p.x &= mmask; p.y &= mmask; p.z &= mmask; p.w &= mmask;
         size_t j = i * 4;
         size_t base = j & ~size_t(mmask);
         uint32_t jl = uint32_t(j) & mmask;
-        Q[base + (p.x & mmask)] = jl;
-        Q[base + (p.y & mmask)] = jl + 1;
-        Q[base + (p.z & mmask)] = jl + 2;
-        Q[base + (p.w & mmask)] = jl + 3;
-    }
-}
-
-// a2: successor g(j) = base + Q[base + (P[j^1] ^ 1)], word = (g(j), j).
-// Two output switches (four outputs) per thread.
-__global__ void __launch_bounds__(kThreads)
-k_build(const uint4 *__restrict__ P4, const uint32_t *__restrict__ Q,
-        ulonglong2 *__restrict__ W2, size_t quads, uint32_t mmask, const uint32_t *__restrict__ gate) {
-    if (gate && *gate == 0u) return;
-    size_t stride = size_t(gridDim.x) * blockDim.x;
-    for (size_t i = size_t(blockIdx.x) * blockDim.x + threadIdx.x; i < quads; i += stride) {
-        uint4 p = __ldg(P4 + i);
-        size_t j = i * 4;
-        size_t base = j & ~size_t(mmask);
-        uint32_t b32 = uint32_t(base);
-        uint32_t g0 = b32 + (__ldg(Q + base + ((p.y & mmask) ^ 1u)) & mmask);
-        uint32_t g1 = b32 + (__ldg(Q + base + ((p.x & mmask) ^ 1u)) & mmask);
-        uint32_t g2 = b32 + (__ldg(Q + base + ((p.w & mmask) ^ 1u)) & mmask);
-        uint32_t g3 = b32 + (__ldg(Q + base + ((p.z & mmask) ^ 1u)) & mmask);
-        uint32_t j32 = uint32_t(j);
-        ulonglong2 a, b;
-        a.x = make_word(g0, j32);
-        a.y = make_word(g1, j32 + 1);
-        b.x = make_word(g2, j32 + 2);
-        b.y = make_word(g3, j32 + 3);
-        W2[2 * i] = a;
-        W2[2 * i + 1] = b;
+        S[2 * i] = make_uint4(p.x, p.y, kUnowned, 0u);
+        S[2 * i + 1] = make_uint4(p.z, p.w, kUnowned, 0u);
+        Q[base + p.x] = jl;
+        Q[base + p.y] = jl + 1;
+        Q[base + p.z] = jl + 2;
+        Q[base + p.w] = jl + 3;
     }
 }
 
@@ -80,37 +63,56 @@ __device__ __forceinline__ unsigned long long jump(unsigned long long w, unsigne
     return (hi << 32) | (t & 0xFFFFFFFFull);
 }
 
-// a3: one in-place pointer-jumping pass.  Four words per thread: two 16-byte
-// loads of the thread's own words, four independent 8-byte gathers.
+// a2 + a3 + a4 + output side of a5 over all outputs of the level, passes
+// separated by grid-wide barriers (cooperative launch).
+//   build : W[j] = (g(j), j), g(j) = base + Q[base + (P[j^1] ^ 1)]
+//   passes: W[j] <- (W[nxt].nxt, min(mn, W[nxt].mn)), in place
+//   last  : even outputs only; colour = leader & 1 -> output-side stage word
 __global__ void __launch_bounds__(kThreads)
-k_jump(unsigned long long *__restrict__ Wd, size_t quads, const uint32_t *__restrict__ gate) {
-    if (gate && *gate == 0u) return;
-    size_t stride = size_t(gridDim.x) * blockDim.x;
+k_full_label(const uint4 *__restrict__ S, const uint32_t *__restrict__ Q,
+             unsigned long long *__restrict__ Wd, size_t total, uint32_t mmask, int passes,
+             BitsLayout L, int out_stage, const uint32_t *__restrict__ gate) {
+    if (gate && *gate == 0u) return;        // same value for every thread of the grid
+    cg::grid_group grid = cg::this_grid();
+    const size_t stride = size_t(gridDim.x) * blockDim.x;
+    const size_t first = size_t(blockIdx.x) * blockDim.x + threadIdx.x;
     ulonglong2 *W2 = reinterpret_cast<ulonglong2 *>(Wd);
-    for (size_t i = size_t(blockIdx.x) * blockDim.x + threadIdx.x; i < quads; i += stride) {
-        ulonglong2 a = __ldcg(W2 + 2 * i);
-        ulonglong2 b = __ldcg(W2 + 2 * i + 1);
-        unsigned long long t0 = __ldcg(Wd + uint32_t(a.x));
-        unsigned long long t1 = __ldcg(Wd + uint32_t(a.y));
-        unsigned long long t2 = __ldcg(Wd + uint32_t(b.x));
-        unsigned long long t3 = __ldcg(Wd + uint32_t(b.y));
-        a.x = jump(a.x, t0);
-        a.y = jump(a.y, t1);
-        b.x = jump(b.x, t2);
-        b.y = jump(b.y, t3);
-        __stcg(W2 + 2 * i, a);
-        __stcg(W2 + 2 * i + 1, b);
-    }
-}
 
-// a3 (last pass) + a4 + out-side half of a5: only the even outputs are
-// needed; colour = leader & 1 goes straight into the output-side stage word.
-__global__ void __launch_bounds__(kThreads)
-k_jump_last(const unsigned long long *__restrict__ Wd, size_t switches, BitsLayout L, int out_stage,
-            const uint32_t *__restrict__ gate) {
-    if (gate && *gate == 0u) return;
-    size_t stride = size_t(gridDim.x) * blockDim.x;
-    for (size_t t = size_t(blockIdx.x) * blockDim.x + threadIdx.x; t < switches; t += stride) {
+    const size_t switches = total / 2;
+    for (size_t t = first; t < switches; t += stride) {
+        uint4 r = __ldg(S + t);
+        size_t j = 2 * t;
+        size_t base = j & ~size_t(mmask);
+        uint32_t b32 = uint32_t(base);
+        uint32_t g0 = b32 + (__ldg(Q + base + ((r.y & mmask) ^ 1u)) & mmask);
+        uint32_t g1 = b32 + (__ldg(Q + base + ((r.x & mmask) ^ 1u)) & mmask);
+        ulonglong2 a;
+        a.x = make_word(g0, uint32_t(j));
+        a.y = make_word(g1, uint32_t(j) + 1u);
+        W2[t] = a;
+    }
+    grid.sync();
+
+    const size_t quads = total / 4;
+    for (int r = 0; r < passes; ++r) {
+        for (size_t i = first; i < quads; i += stride) {
+            ulonglong2 a = __ldcg(W2 + 2 * i);
+            ulonglong2 b = __ldcg(W2 + 2 * i + 1);
+            unsigned long long t0 = __ldcg(Wd + uint32_t(a.x));
+            unsigned long long t1 = __ldcg(Wd + uint32_t(a.y));
+            unsigned long long t2 = __ldcg(Wd + uint32_t(b.x));
+            unsigned long long t3 = __ldcg(Wd + uint32_t(b.y));
+            a.x = jump(a.x, t0);
+            a.y = jump(a.y, t1);
+            b.x = jump(b.x, t2);
+            b.y = jump(b.y, t3);
+            __stcg(W2 + 2 * i, a);
+            __stcg(W2 + 2 * i + 1, b);
+        }
+        grid.sync();
+    }
+
+    for (size_t t = first; t < switches; t += stride) {
         unsigned long long w = __ldcg(Wd + 2 * t);
         unsigned long long v = __ldcg(Wd + uint32_t(w));
         uint32_t mn = uint32_t(jump(w, v) >> 32);
@@ -119,9 +121,12 @@ k_jump_last(const unsigned long long *__restrict__ Wd, size_t switches, BitsLayo
     }
 }
 
-// in-side half of a5 + a6: input-side stage word, P' and Q'.
+// in-side half of a5 + a6: input-side stage word, next level's records and Q'.
+// Position tl of the upper half-block takes P[2t or 2t+1] >> 1 of switch tl,
+// so two neighbouring threads hold the two values of one record of the next
+// level: they exchange them with a shuffle and store whole records.
 __global__ void __launch_bounds__(kThreads)
-k_split(const uint2 *__restrict__ P2, const uint2 *__restrict__ Q2, uint32_t *__restrict__ Pn,
+k_split(const uint4 *__restrict__ S, const uint2 *__restrict__ Q2, uint4 *__restrict__ Sn,
         uint32_t *__restrict__ Qn, size_t switches, uint32_t mmask, BitsLayout L, int in_stage,
         int out_stage) {
     size_t stride = size_t(gridDim.x) * blockDim.x;
@@ -129,13 +134,17 @@ k_split(const uint2 *__restrict__ P2, const uint2 *__restrict__ Q2, uint32_t *__
     for (size_t t = size_t(blockIdx.x) * blockDim.x + threadIdx.x; t < switches; t += stride) {
         size_t base = (2 * t) & ~size_t(mmask);
         uint32_t tl = uint32_t(t - base / 2);
-        uint2 p = __ldg(P2 + t);
-        uint2 q = __ldg(Q2 + t);
-        p.x &= mmask; p.y &= mmask; q.x &= mmask; q.y &= mmask;
+        uint4 r = __ldcs(S + t);
+        uint2 q = __ldcs(Q2 + t);
+        r.x &= mmask; r.y &= mmask; q.x &= mmask; q.y &= mmask;
         // colour of output 2t
         uint32_t c = (L.bits[L.word(out_stage, t >> 5)] >> (t & 31)) & 1u;
-        Pn[base + c * H + tl] = p.x >> 1;
-        Pn[base + (1u - c) * H + tl] = p.y >> 1;
+        uint32_t up = (c ? r.y : r.x) >> 1, lo = (c ? r.x : r.y) >> 1;
+        uint32_t got = __shfl_xor_sync(0xFFFFFFFFu, (tl & 1u) ? up : lo, 1);
+        if (tl & 1u)
+            Sn[(base >> 1) + (H >> 1) + (tl >> 1)] = make_uint4(got, lo, kUnowned, 0u);
+        else
+            Sn[(base >> 1) + (tl >> 1)] = make_uint4(up, got, kUnowned, 0u);
         // colour of the output fed by input 2t
         size_t o = base + q.x;
         uint32_t cin = ((L.bits[L.word(out_stage, o >> 6)] >> ((o >> 1) & 31)) & 1u) ^ (q.x & 1u);
@@ -160,42 +169,60 @@ k_validate(const uint32_t *__restrict__ perm, size_t total, uint32_t nmask,
     }
 }
 
+// CTAs of k_full_label that are resident together on the current device.
+int cooperative_grid(int *out) {
+    constexpr int kMaxDev = 64;
+    static int cached[kMaxDev] = {};
+    int dev = 0;
+    BENES_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDev) return BENES_ERR_CUDA;
+    if (!cached[dev]) {
+        int sms = 0, per_sm = 0, coop = 0;
+        BENES_CUDA_TRY(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev));
+        if (!coop) return BENES_ERR_CUDA;
+        BENES_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+        BENES_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_full_label, kThreads, 0));
+        if (sms < 1 || per_sm < 1) return BENES_ERR_CUDA;
+        cached[dev] = sms * per_sm;
+    }
+    *out = cached[dev];
+    return BENES_OK;
+}
+
 }  // namespace
 
-int launch_inverse(const uint32_t *P, uint32_t *Q, size_t total, int log2m, cudaStream_t s) {
+int launch_inverse(const uint32_t *perm, uint4 *S, uint32_t *Q, size_t total, int log2m,
+                   cudaStream_t s) {
     size_t quads = total / 4;
-    k_inverse<<<grid_for(quads), kThreads, 0, s>>>(reinterpret_cast<const uint4 *>(P), Q, quads,
-                                                   (1u << log2m) - 1u);
+    k_inverse<<<grid_for(quads), kThreads, 0, s>>>(reinterpret_cast<const uint4 *>(perm), S, Q,
+                                                   quads, (1u << log2m) - 1u);
     return launch_status();
 }
 
-int launch_build(const uint32_t *P, const uint32_t *Q, unsigned long long *Wd, size_t total,
-                 int log2m, const uint32_t *gate, cudaStream_t s) {
-    size_t quads = total / 4;
-    k_build<<<grid_for(quads), kThreads, 0, s>>>(reinterpret_cast<const uint4 *>(P), Q,
-                                                 reinterpret_cast<ulonglong2 *>(Wd), quads,
-                                                 (1u << log2m) - 1u, gate);
+int launch_full_label(const uint4 *S, const uint32_t *Q, unsigned long long *Wd, size_t total,
+                      int log2m, BitsLayout L, int out_stage, const uint32_t *gate,
+                      cudaStream_t s) {
+    int grid = 0;
+    int rc = cooperative_grid(&grid);
+    if (rc) return rc;
+    size_t need = (total / 2 + kThreads - 1) / kThreads;
+    if (size_t(grid) > need) grid = int(need);
+    uint32_t mmask = (1u << log2m) - 1u;
+    int passes = log2m - 2;
+    void *args[] = {(void *)&S, (void *)&Q, (void *)&Wd, (void *)&total, (void *)&mmask,
+                    (void *)&passes, (void *)&L, (void *)&out_stage, (void *)&gate};
+    if (cudaLaunchCooperativeKernel((const void *)k_full_label, dim3(grid), dim3(kThreads), args, 0,
+                                    s) != cudaSuccess) {
+        cudaGetLastError();
+        return BENES_ERR_CUDA;
+    }
     return launch_status();
 }
 
-int launch_jump(unsigned long long *Wd, size_t total, const uint32_t *gate, cudaStream_t s) {
-    size_t quads = total / 4;
-    k_jump<<<grid_for(quads), kThreads, 0, s>>>(Wd, quads, gate);
-    return launch_status();
-}
-
-int launch_jump_last(const unsigned long long *Wd, size_t total, BitsLayout L, int out_stage,
-                     const uint32_t *gate, cudaStream_t s) {
-    size_t switches = total / 2;
-    k_jump_last<<<grid_for(switches), kThreads, 0, s>>>(Wd, switches, L, out_stage, gate);
-    return launch_status();
-}
-
-int launch_split(const uint32_t *P, const uint32_t *Q, uint32_t *Pn, uint32_t *Qn, size_t total,
+int launch_split(const uint4 *S, const uint32_t *Q, uint4 *Sn, uint32_t *Qn, size_t total,
                  int log2m, BitsLayout L, int in_stage, int out_stage, cudaStream_t s) {
     size_t switches = total / 2;
-    k_split<<<grid_for(switches), kThreads, 0, s>>>(reinterpret_cast<const uint2 *>(P),
-                                                    reinterpret_cast<const uint2 *>(Q), Pn, Qn,
+    k_split<<<grid_for(switches), kThreads, 0, s>>>(S, reinterpret_cast<const uint2 *>(Q), Sn, Qn,
                                                     switches, (1u << log2m) - 1u, L, in_stage,
                                                     out_stage);
     return launch_status();

@@ -1,29 +1,38 @@
 // Work-efficient loop labelling for the HBM levels: ruler sampling.
 //
 // Pointer jumping over all outputs costs O(M log M) random accesses per level.
-// Here only a sample of the outputs (the "rulers") is labelled by pointer
-// jumping; everything else is reached by one sequential walk per ruler:
+// Here every output switch is visited ONCE per level:
 //
 //   1. Switches are cut into groups of k = 2^kappa consecutive switches; a hash
 //      of the group number picks one RULER switch per group.  Both outputs of
 //      a ruler switch are ruler outputs; ruler output rho = 2*group + (j & 1).
 //   2. k_walk: one thread per ruler output follows the successor
-//      g(j) = base + Q[base + (P[j^1] ^ 1)] until it meets the next ruler
-//      output.  It records (next ruler, smallest index seen) as one 64-bit
-//      word of the contracted list and stamps its id on every even output it
-//      passes ("owner" of the switch).  Every output lies on exactly one such
-//      segment, so the walks cost O(M) in total.
-//   3. The contracted list (T/k words, cache resident) is labelled by the
-//      ordinary in-place pointer-jumping pass: afterwards a ruler's word holds
-//      the minimum of its whole g-cycle.
-//   4. k_colour: colour of output 2t = parity of the cycle minimum of its
-//      owner.  A switch nobody stamped lies on a loop without ruler; such
-//      loops are short (probability (1-1/k)^length) and the thread walks the
-//      cycle itself.
+//      g(j) = base + Q[base + (P[j^1] ^ 1)].  The g-cycle through output j
+//      and the g-cycle through j^1 are mirror images (g(g(j)^1) = j^1), so the
+//      walker that leaves ruler switch T forwards and the walker that leaves
+//      the next ruler switch T' backwards run over the same switches from the
+//      two ends.  Each claims the switches it reaches with a compare-and-swap
+//      on the record's owner field and stops at the first switch the other one
+//      owns: together they touch every switch of the segment once.  A walker
+//      keeps the smallest output index on its own side of the switches it
+//      claimed (fwd), the smallest on the far side (part), and its partner
+//      (peer).  The claim stores (walker, side of arrival).
+//   3. k_combine: the segment of walker rho ends at ruler output peer^1 and
+//      its minimum is min(fwd[rho], part[peer]): one 64-bit (next, min) word
+//      per ruler output -- the contracted list.
+//   4. The contracted list is labelled with the minimum of every cycle:
+//      lists of up to 2^14 words per block in one CTA's shared memory, longer
+//      ones by sampling again (one ruler per 16 words, plain one-directional
+//      walks: the list is cache resident).
+//   5. k_colour: output 2t lies on its owner's cycle if the owner arrived on
+//      the even side, else on the mirror cycle, which has the other colour:
+//      colour = (cycle minimum of the owner & 1) ^ side.  A switch nobody
+//      claimed lies on a loop without ruler; such loops are short
+//      (probability (1-1/k)^length) and the thread walks the cycle itself.
 //
-// Both walks give up after `cap` hops and raise a per-level flag; the flag
-// gates the full pointer-jumping kernels of route_levels.cu, which then
-// relabel the level.  So the result never depends on the sampling.
+// Every walk gives up after `cap` hops and raises the level's gate; the gate
+// opens the full pointer-jumping kernel of route_levels.cu, which relabels the
+// level.  So the result never depends on the sampling.
 #include "common.cuh"
 
 namespace benes {
@@ -31,7 +40,8 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kSMs = 148;
-constexpr uint32_t kUnowned = 0xFFFFFFFFu;
+constexpr int kListThreads = 1024;
+constexpr int kListPer = (1 << kListSmemLog2) / kListThreads;   // words per thread, at most
 
 __device__ __forceinline__ uint32_t ruler_slot(uint32_t group, uint32_t salt, uint32_t kmask) {
     uint32_t h = group * 0x9E3779B1u + salt;
@@ -41,101 +51,327 @@ __device__ __forceinline__ uint32_t ruler_slot(uint32_t group, uint32_t salt, ui
     return h & kmask;
 }
 
-__device__ __forceinline__ unsigned long long make_word(uint32_t nxt, uint32_t mn) {
-    return (static_cast<unsigned long long>(mn) << 32) | nxt;
+__device__ __forceinline__ bool gate_raised(const uint32_t *gate) {
+    return *reinterpret_cast<const volatile uint32_t *>(gate) != 0u;
 }
 
 // Step 2.  rulers = T / k threads, launched in index order so that the blocks
 // being walked at any moment are neighbours in memory.
 __global__ void __launch_bounds__(kThreads)
-k_walk(const uint32_t *__restrict__ P, const uint32_t *__restrict__ Q, uint32_t *__restrict__ owner,
-       unsigned long long *__restrict__ Wc, uint32_t rulers, uint32_t mmask, int kappa,
-       uint32_t salt, uint32_t cap, uint32_t *__restrict__ gate) {
+k_walk(uint4 *__restrict__ S, const uint32_t *__restrict__ Q, uint4 *__restrict__ rec,
+       uint32_t rulers, uint32_t mmask, int kappa, uint32_t salt, uint32_t cap,
+       uint32_t *__restrict__ gate) {
     const uint32_t rho = blockIdx.x * kThreads + threadIdx.x;
     if (rho >= rulers) return;
     const uint32_t kmask = (1u << kappa) - 1u;
-    const uint32_t group = rho >> 1;
+    const uint32_t group = rho >> 1, side0 = rho & 1u;
     const uint32_t t0 = (group << kappa) | ruler_slot(group, salt, kmask);
-    uint32_t j = 2u * t0 + (rho & 1u);
+    uint32_t j = 2u * t0 + side0;
     const uint32_t base = j & ~mmask;
-    uint32_t mn = j, nxt = rho, hops = 0;
-    if (!(rho & 1u)) owner[t0] = rho;
+    uint32_t fwd = j, part = kUnowned, peer = rho ^ 1u, hops = 0;
+    uint4 r = __ldcg(S + t0);
+    // the ruler switch belongs to its even-side walker (nobody else claims it)
+    if (!side0) reinterpret_cast<uint32_t *>(S + t0)[2] = rho << 1;
+    uint32_t p = (side0 ? r.x : r.y) & mmask;                     // P[j^1]
+    uint32_t q = __ldcg(Q + base + (p ^ 1u)) & mmask;
     for (;;) {
-        uint32_t p = __ldg(P + (j ^ 1u)) & mmask;
-        j = base + (__ldg(Q + base + (p ^ 1u)) & mmask);
-        uint32_t t = j >> 1, g = t >> kappa;
-        if ((t & kmask) == ruler_slot(g, salt, kmask)) {
-            nxt = 2u * g + (j & 1u);
+        j = base + q;
+        const uint32_t t = j >> 1, side = j & 1u, g = t >> kappa;
+        if ((t & kmask) == ruler_slot(g, salt, kmask)) {          // reached the next ruler
+            peer = (2u * g + side) ^ 1u;
             break;
         }
-        if (++hops > cap) {         // give up: the word stays a self loop
+        if (++hops > cap) {
             *gate = 1u;
             break;
         }
-        // somebody else gave up: the level is relabelled anyway
-        if ((hops & 63u) == 0u && *reinterpret_cast<volatile uint32_t *>(gate)) break;
-        mn = min(mn, j);
-        if (!(j & 1u)) owner[t] = rho;
+        if ((hops & 63u) == 0u && gate_raised(gate)) break;       // the level is relabelled anyway
+        r = __ldcg(S + t);
+        p = (side ? r.x : r.y) & mmask;
+        // next hop's gather, issued before the claim is known (harmless if we stop)
+        const uint32_t qn = __ldcg(Q + base + (p ^ 1u)) & mmask;
+        uint32_t prev = r.z;
+        if (prev == kUnowned)
+            prev = atomicCAS(reinterpret_cast<uint32_t *>(S + t) + 2, kUnowned, (rho << 1) | side);
+        if (prev != kUnowned) {                                   // met the walker from the other end
+            peer = prev >> 1;
+            break;
+        }
+        fwd = min(fwd, j);
+        part = min(part, j ^ 1u);
+        q = qn;
     }
-    Wc[rho] = make_word(nxt, mn);
+    rec[rho] = make_uint4(fwd, part, peer, 0u);
 }
 
-// Step 4 + output side of the level's switches.
+// Step 3.
 __global__ void __launch_bounds__(kThreads)
-k_colour(const uint32_t *__restrict__ P, const uint32_t *__restrict__ Q,
-         const uint32_t *__restrict__ owner, const unsigned long long *__restrict__ Wc,
-         size_t switches, uint32_t mmask, BitsLayout L, int out_stage, uint32_t cap,
-         uint32_t *__restrict__ gate) {
+k_combine(const uint4 *__restrict__ rec, unsigned long long *__restrict__ W, uint32_t rulers) {
+    const uint32_t rho = blockIdx.x * kThreads + threadIdx.x;
+    if (rho >= rulers) return;
+    const uint4 a = rec[rho];
+    const uint32_t peer = a.z < rulers ? a.z : rho;
+    const uint4 b = __ldg(rec + peer);
+    W[rho] = make_word(peer ^ 1u, min(a.x, b.y));
+}
+
+// Step 4, sampling a list: one ruler per 16 words; a thread walks from its
+// ruler to the next one, stamps itself on the words it passes and writes one
+// word (next ruler, minimum) of the 16 times shorter list.
+__global__ void __launch_bounds__(kThreads)
+k_list_walk(const unsigned long long *__restrict__ W, uint32_t *__restrict__ owner,
+            unsigned long long *__restrict__ W2, uint32_t rulers, uint32_t wmask, uint32_t salt,
+            uint32_t cap, uint32_t *__restrict__ gate) {
+    const uint32_t rho = blockIdx.x * kThreads + threadIdx.x;
+    if (rho >= rulers) return;
+    constexpr uint32_t kmask = (1u << kListKappa) - 1u;
+    uint32_t e = (rho << kListKappa) | ruler_slot(rho, salt, kmask);
+    unsigned long long w = __ldcg(W + e);
+    uint32_t mn = uint32_t(w >> 32), nxt = rho, hops = 0;
+    owner[e] = rho;
+    for (;;) {
+        e = uint32_t(w) & wmask;
+        const uint32_t g = e >> kListKappa;
+        if ((e & kmask) == ruler_slot(g, salt, kmask)) {
+            nxt = g;
+            break;
+        }
+        if (++hops > cap) {
+            *gate = 1u;
+            break;
+        }
+        if ((hops & 63u) == 0u && gate_raised(gate)) break;
+        w = __ldcg(W + e);
+        mn = min(mn, uint32_t(w >> 32));
+        owner[e] = rho;
+    }
+    W2[rho] = make_word(nxt, mn);
+}
+
+// Step 4, back from a sampled list: every word takes the cycle minimum of its
+// owner (and hands the owner slot back as kUnowned); a word without owner
+// walks its own cycle.
+__global__ void __launch_bounds__(kThreads)
+k_list_resolve(unsigned long long *__restrict__ W, uint32_t *__restrict__ owner,
+               const unsigned long long *__restrict__ W2, uint32_t count, uint32_t wmask,
+               uint32_t cap, uint32_t *__restrict__ gate) {
+    const uint32_t e0 = blockIdx.x * kThreads + threadIdx.x;
+    if (e0 >= count) return;
+    const uint32_t o = owner[e0];
+    unsigned long long w = __ldcg(W + e0);
+    uint32_t mn;
+    if (o != kUnowned) {
+        mn = uint32_t(__ldcg(W2 + o) >> 32);
+        owner[e0] = kUnowned;
+    } else {
+        // words rewritten meanwhile hold the minimum of this same cycle: harmless
+        mn = uint32_t(w >> 32);
+        uint32_t e = uint32_t(w) & wmask, hops = 0;
+        while (e != e0) {
+            if (++hops > cap) {
+                *gate = 1u;
+                break;
+            }
+            const unsigned long long v = __ldcg(W + e);
+            mn = min(mn, uint32_t(v >> 32));
+            e = uint32_t(v) & wmask;
+        }
+    }
+    __stcg(W + e0, make_word(uint32_t(w), mn));
+}
+
+// Step 4, the end of the recursion: one CTA labels one block's list of
+// 2^log2b words in shared memory by synchronous pointer jumping (new words are
+// held in registers across the barrier).  A cycle has at most 2^log2b words
+// (a list sampled from a list need not split evenly between a cycle and its
+// mirror image), hence log2b passes.
+__global__ void __launch_bounds__(kListThreads)
+k_list_label(unsigned long long *__restrict__ W, int log2b) {
+    extern __shared__ unsigned long long sm[];
+    const uint32_t B = 1u << log2b, bmask = B - 1u;
+    const size_t base = size_t(blockIdx.x) << log2b;
+    const uint32_t T = blockDim.x, tid = threadIdx.x;
+    for (uint32_t e = tid; e < B; e += T) {
+        unsigned long long w = __ldcs(W + base + e);
+        sm[e] = make_word(uint32_t(w) & bmask, uint32_t(w >> 32));
+    }
+    __syncthreads();
+    unsigned long long v[kListPer];
+    for (int pass = 0; pass < log2b; ++pass) {
+#pragma unroll
+        for (int i = 0; i < kListPer; ++i) {
+            const uint32_t e = tid + uint32_t(i) * T;
+            if (e < B) {
+                const unsigned long long w = sm[e];
+                const unsigned long long t = sm[uint32_t(w)];
+                v[i] = make_word(uint32_t(t), min(uint32_t(w >> 32), uint32_t(t >> 32)));
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int i = 0; i < kListPer; ++i) {
+            const uint32_t e = tid + uint32_t(i) * T;
+            if (e < B) sm[e] = v[i];
+        }
+        __syncthreads();
+    }
+    for (uint32_t e = tid; e < B; e += T) {
+        const unsigned long long w = sm[e];
+        W[base + e] = make_word(uint32_t(base) + uint32_t(w), uint32_t(w >> 32));
+    }
+}
+
+// Step 5 + output side of the level's switches.
+__global__ void __launch_bounds__(kThreads)
+k_colour(const uint4 *__restrict__ S, const uint32_t *__restrict__ Q,
+         const unsigned long long *__restrict__ W, size_t switches, uint32_t rulers, uint32_t mmask,
+         BitsLayout L, int out_stage, uint32_t cap, uint32_t *__restrict__ gate) {
     const size_t stride = size_t(gridDim.x) * blockDim.x;
     for (size_t t = size_t(blockIdx.x) * blockDim.x + threadIdx.x; t < switches; t += stride) {
-        uint32_t o = __ldcs(owner + t);
-        uint32_t mn;
-        if (o != kUnowned) {
-            mn = uint32_t(__ldg(Wc + o) >> 32);
+        const uint32_t code = __ldcs(reinterpret_cast<const uint32_t *>(S + t) + 2);
+        uint32_t c;
+        if (code != kUnowned) {
+            const uint32_t rho = code >> 1;
+            c = (uint32_t(__ldg(W + (rho < rulers ? rho : 0u)) >> 32) ^ code) & 1u;
         } else {
             // loop without ruler: walk the g-cycle of output 2t
             const uint32_t j0 = uint32_t(2 * t);
             const uint32_t base = j0 & ~mmask;
-            uint32_t j = j0, hops = 0;
-            mn = j0;
+            uint32_t j = j0, mn = j0, hops = 0;
             for (;;) {
-                uint32_t p = __ldg(P + (j ^ 1u)) & mmask;
+                const uint32_t p = rec_p(S, j ^ 1u) & mmask;
                 j = base + (__ldg(Q + base + (p ^ 1u)) & mmask);
                 if (j == j0) break;
                 if (++hops > cap) {
                     *gate = 1u;
                     break;
                 }
-                if ((hops & 63u) == 0u && *reinterpret_cast<volatile uint32_t *>(gate)) break;
+                if ((hops & 63u) == 0u && gate_raised(gate)) break;
                 mn = min(mn, j);
             }
+            c = mn & 1u;
         }
-        uint32_t word = __ballot_sync(0xFFFFFFFFu, mn & 1u);
+        const uint32_t word = __ballot_sync(0xFFFFFFFFu, c);
         if ((threadIdx.x & 31) == 0) L.bits[L.word(out_stage, t >> 5)] = word;
     }
 }
 
-}  // namespace
+inline size_t align256(size_t v) { return (v + 255) & ~size_t(255); }
+constexpr int kMaxLists = 5;
 
-int launch_walk(const uint32_t *P, const uint32_t *Q, uint32_t *owner, unsigned long long *Wc,
-                size_t total, int log2m, int kappa, uint32_t salt, uint32_t cap, uint32_t *gate,
-                cudaStream_t s) {
-    const size_t rulers = total >> kappa;
-    const unsigned grid = unsigned((rulers + kThreads - 1) / kThreads);
-    k_walk<<<grid, kThreads, 0, s>>>(P, Q, owner, Wc, uint32_t(rulers), (1u << log2m) - 1u, kappa,
-                                     salt, cap, gate);
-    return launch_status();
+// Number of times the list of a block with 2^beta words is sampled again.
+inline int list_depth(int beta) {
+    int d = 0;
+    while (beta > kListSmemLog2 && d < kMaxLists - 1) {
+        beta -= kListKappa;
+        ++d;
+    }
+    return d;
 }
 
-int launch_colour(const uint32_t *P, const uint32_t *Q, const uint32_t *owner,
-                  const unsigned long long *Wc, size_t total, int log2m, BitsLayout L,
-                  int out_stage, uint32_t cap, uint32_t *gate, cudaStream_t s) {
-    const size_t switches = total / 2;
-    size_t blocks = (switches + kThreads - 1) / kThreads;
-    const size_t capb = size_t(kSMs) * 8;
-    k_colour<<<unsigned(blocks < capb ? blocks : capb), kThreads, 0, s>>>(
-        P, Q, owner, Wc, switches, (1u << log2m) - 1u, L, out_stage, cap, gate);
-    return launch_status();
+}  // namespace
+
+// Scratch: walk records, the contracted lists and the owners of every list
+// that may be sampled again.  Sized for the largest level (log2m = 30).
+size_t sampled_scratch_bytes(size_t total, int kappa) {
+    size_t R = total >> kappa, bytes = align256(R * 16);
+    for (int i = 0; i < kMaxLists; ++i) {
+        size_t c = R >> (kListKappa * i);
+        if (c < 4) c = 4;
+        bytes += align256(c * 8) + align256(c * 4);
+    }
+    return bytes;
+}
+
+void sampled_scratch_carve(char *base, size_t total, int kappa, SampledScratch *out) {
+    size_t R = total >> kappa, off = 0;
+    out->rec = reinterpret_cast<uint4 *>(base);
+    off += align256(R * 16);
+    for (int i = 0; i < kMaxLists; ++i) {
+        size_t c = R >> (kListKappa * i);
+        if (c < 4) c = 4;
+        out->list[i] = reinterpret_cast<unsigned long long *>(base + off);
+        off += align256(c * 8);
+        out->owner[i] = reinterpret_cast<uint32_t *>(base + off);
+        off += align256(c * 4);
+    }
+}
+
+int sampled_scratch_reset(const SampledScratch &sc, size_t total, int kappa, cudaStream_t s) {
+    size_t R = total >> kappa;
+    for (int i = 0; i < kMaxLists - 1; ++i) {
+        size_t c = R >> (kListKappa * i);
+        if (c < 4) c = 4;
+        BENES_CUDA_TRY(cudaMemsetAsync(sc.owner[i], 0xFF, c * 4, s));
+    }
+    return BENES_OK;
+}
+
+int sampled_label(uint4 *S, const uint32_t *Q, const SampledScratch &sc, size_t total, int log2m,
+                  int kappa, uint32_t salt, uint32_t cap, BitsLayout L, int out_stage,
+                  uint32_t *gate, cudaStream_t s) {
+    const uint32_t mmask = (1u << log2m) - 1u;
+    const uint32_t R = uint32_t(total >> kappa);
+    const unsigned rgrid = (R + kThreads - 1) / kThreads;
+    {
+        ProfileScope ps(kWalk, s);
+        k_walk<<<rgrid, kThreads, 0, s>>>(S, Q, sc.rec, R, mmask, kappa, salt, cap, gate);
+        int rc = launch_status();
+        if (rc) return rc;
+    }
+    {
+        ProfileScope ps(kCombine, s);
+        k_combine<<<rgrid, kThreads, 0, s>>>(sc.rec, sc.list[0], R);
+        int rc = launch_status();
+        if (rc) return rc;
+    }
+    // label the contracted list: sample it until a block's list fits one CTA
+    int beta = log2m - kappa;
+    const int depth = list_depth(beta);
+    uint32_t count = R;
+    for (int d = 0; d < depth; ++d) {
+        ProfileScope ps(kListWalk, s);
+        const uint32_t next = count >> kListKappa;
+        k_list_walk<<<(next + kThreads - 1) / kThreads, kThreads, 0, s>>>(
+            sc.list[d], sc.owner[d], sc.list[d + 1], next, count - 1u, salt * 7u + uint32_t(d) + 1u,
+            cap, gate);
+        int rc = launch_status();
+        if (rc) return rc;
+        count = next;
+        beta -= kListKappa;
+    }
+    {
+        ProfileScope ps(kListLabel, s);
+        static bool configured = false;
+        if (!configured) {
+            BENES_CUDA_TRY(cudaFuncSetAttribute(k_list_label, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                (1 << kListSmemLog2) * 8));
+            configured = true;
+        }
+        if (beta > kListSmemLog2) return BENES_ERR_BADARG;
+        const uint32_t B = 1u << beta;
+        const unsigned threads = B < unsigned(kListThreads) ? (B < 32u ? 32u : B) : unsigned(kListThreads);
+        k_list_label<<<count >> beta, threads, size_t(B) * 8, s>>>(sc.list[depth], beta);
+        int rc = launch_status();
+        if (rc) return rc;
+    }
+    for (int d = depth - 1; d >= 0; --d) {
+        ProfileScope ps(kListResolve, s);
+        const uint32_t c = R >> (kListKappa * d);
+        k_list_resolve<<<(c + kThreads - 1) / kThreads, kThreads, 0, s>>>(
+            sc.list[d], sc.owner[d], sc.list[d + 1], c, c - 1u, cap, gate);
+        int rc = launch_status();
+        if (rc) return rc;
+    }
+    {
+        ProfileScope ps(kColour, s);
+        const size_t switches = total / 2;
+        size_t blocks = (switches + kThreads - 1) / kThreads;
+        const size_t capb = size_t(kSMs) * 8;
+        k_colour<<<unsigned(blocks < capb ? blocks : capb), kThreads, 0, s>>>(
+            S, Q, sc.list[0], switches, R, mmask, L, out_stage, cap, gate);
+        return launch_status();
+    }
 }
 
 }  // namespace benes
