@@ -306,6 +306,10 @@ def run_gpu(args):
         for k in range(binding.PROFILE_KINDS):
             cnt, ms = binding.benes_profile_read(k)
             kinds[binding.benes_profile_kind_name(k)] = {"launches": cnt, "ms": ms}
+        spans = binding.benes_profile_spans()
+        per_level = {}
+        for kname, _, ms in spans[:len(spans) // args.steps]:       # first timed step
+            per_level.setdefault(kname, []).append(round(ms, 3))
         binding.benes_profile_reset()
         clocks = sampler.stop() if rank == 0 else None
 
@@ -388,6 +392,8 @@ def run_gpu(args):
                           "route_elements_per_s": elems / (route_ms * 1e-3),
                           "apply_elements_per_s": elems / (apply_ms * 1e-3),
                           "kernel_ms_per_step": {k: v["ms"] / args.steps for k, v in kinds.items()},
+                          "first_step_ms_by_level": {k: v for k, v in per_level.items()
+                                                     if k in ("walk", "colour", "split", "list_label", "list_walk")},
                           "kernel_launches_per_step": {k: v["launches"] // args.steps for k, v in kinds.items()}},
         }
         if world == 1 and not args.no_cpu_baseline:

@@ -73,7 +73,7 @@ int benes_route(const uint32_t *perm, int log2n, int batch, uint32_t *switch_bit
                 benes_stream_t stream);
 
 /*
- * Route a payload of 4-byte elements through the network, one pass per stage:
+ * Route a payload of 4-byte elements through the 2n-1 stages of the network:
  * out[b][j] = in[b][pi_b[j]] when switch_bits came from benes_route(pi).
  *   in, out : batch x N elements; must not overlap; in is read only.
  */
@@ -153,11 +153,15 @@ int benes_validate_perm(const uint32_t *perm, int log2n, int batch, benes_stream
  *       sequential walks between rulers.  The result is identical either way.
  *   BENES_OPT_WALK_CAP : hops (1 .. 2^24, default 2^14) after which a walk gives
  *       up; a level in which that happens is relabelled by full pointer jumping.
+ *   BENES_OPT_APPLY_FUSED : 1 (default) = benes_apply / benes_apply_ex run up to
+ *       25 stages per pass over the payload in shared memory; 0 = one stage per
+ *       pass.  Same result.
  * benes_set_option returns BENES_OK or BENES_ERR_BADARG; benes_get_option
  * returns the value, or BENES_ERR_BADARG for an unknown key.
  */
 #define BENES_OPT_SAMPLE_LOG2K 0
 #define BENES_OPT_WALK_CAP 1
+#define BENES_OPT_APPLY_FUSED 2
 int benes_set_option(int key, int value);
 int benes_get_option(int key);
 
@@ -180,6 +184,10 @@ unsigned long long benes_launch_count(void);
 int benes_profile_enable(int on);
 int benes_profile_reset(void);
 int benes_profile_read(int kind, unsigned long long *launches, double *milliseconds);
+/* The index-th timed group since the last reset, in launch order (one group per
+ * kind per recursion level): its kind, launches and device time.
+ * BENES_ERR_BADARG once index is past the last group. */
+int benes_profile_span(int index, int *kind, unsigned long long *launches, double *milliseconds);
 const char *benes_profile_kind_name(int kind);
 
 /* Largest block size (log2) finished inside one CTA by the fused kernel. */

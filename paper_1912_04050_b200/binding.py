@@ -45,6 +45,8 @@ SYMBOLS = {
     "benes_profile_enable": (_i, [_i]),
     "benes_profile_reset": (_i, []),
     "benes_profile_read": (_i, [_i, ctypes.POINTER(ctypes.c_ulonglong), ctypes.POINTER(ctypes.c_double)]),
+    "benes_profile_span": (_i, [_i, ctypes.POINTER(_i), ctypes.POINTER(ctypes.c_ulonglong),
+                                ctypes.POINTER(ctypes.c_double)]),
     "benes_profile_kind_name": (ctypes.c_char_p, [_i]),
     "benes_fused_log2m": (_i, []),
     "benes_status_string": (ctypes.c_char_p, [_i]),
@@ -185,6 +187,7 @@ def benes_launch_count() -> int:
 PROFILE_KINDS = 12
 OPT_SAMPLE_LOG2K = 0
 OPT_WALK_CAP = 1
+OPT_APPLY_FUSED = 2
 
 
 def benes_set_option(key: int, value: int) -> None:
@@ -211,6 +214,16 @@ def benes_profile_read(kind: int):
     n, ms = ctypes.c_ulonglong(0), ctypes.c_double(0.0)
     _check(load().benes_profile_read(kind, ctypes.byref(n), ctypes.byref(ms)), "benes_profile_read")
     return n.value, ms.value
+
+
+def benes_profile_spans():
+    """[(kind name, launches, milliseconds), ...] of every timed group since the last reset."""
+    out, i = [], 0
+    k, n, ms = ctypes.c_int(0), ctypes.c_ulonglong(0), ctypes.c_double(0.0)
+    while load().benes_profile_span(i, ctypes.byref(k), ctypes.byref(n), ctypes.byref(ms)) == BENES_OK:
+        out.append((benes_profile_kind_name(k.value), n.value, ms.value))
+        i += 1
+    return out
 
 
 def benes_profile_kind_name(kind: int) -> str:

@@ -1,0 +1,261 @@
+// Payload apply over several stages per pass.
+//
+// One stage per kernel moves the whole payload through HBM 2n-1 times.  Here a
+// CTA keeps 2^13 elements in shared memory and runs many stages on them:
+//
+//   inner kernel : every block of 2^b elements (b = min(n, 13)) of level n-b
+//                  is closed under the 2b-1 innermost stages (input side of
+//                  levels n-b .. n-2, middle, output side back up to n-b);
+//   outer kernels: k <= 7 consecutive input-side stages of levels l0..l0+k-1
+//                  send a contiguous chunk of 2^k * T elements of a level-l0
+//                  block to 2^k runs of T consecutive positions (one run per
+//                  path through the k switches), so a CTA reads one chunk,
+//                  runs k stages and writes 2^k coalesced runs; the
+//                  output-side kernel is the mirror image.
+//
+// In shared memory nothing moves except through the switches.  Element "slot"
+// u of a chunk keeps, in its low bits, the outcomes of the stages done so far
+// (bit i = 1 if the element left stage l0+i through the lower output) and in
+// its high bits the part of its position the remaining stages still act on:
+// stage l0+i pairs slots u and u | (1 << i), and a crossed switch swaps them.
+// The true position after i stages is
+//     (bit-reversed low i bits of u) << (m0 - i)  +  (X0 >> i) + (u >> i),
+// m0 = log2 of the level-l0 block size, X0 = offset of the chunk in that
+// block; this gives both the switch index of a pair and where a slot is
+// written at the end.  The output side reads the same relation backwards.
+//
+// A thread holds 8 slots (3 slot bits) in registers and runs 3 stages between
+// two barriers.
+#include "common.cuh"
+
+namespace benes {
+namespace {
+
+constexpr int kChunkLog2 = 13;               // elements per CTA
+constexpr int kChunk = 1 << kChunkLog2;
+constexpr int kRound = 3;                    // stages between barriers
+constexpr int kApplyThreads = kChunk >> kRound;
+
+__device__ __forceinline__ uint32_t phys(uint32_t u) { return u + (u >> 5); }
+constexpr int kSmemElems = kChunk + (kChunk >> 5);
+
+__device__ __forceinline__ uint32_t rev_bits(uint32_t v, int i) {
+    return i ? (__brev(v) >> (32 - i)) : 0u;
+}
+
+struct Geometry {
+    const uint32_t *bits_p;   // switch words of this permutation
+    uint32_t stage_w;         // words per stage
+    uint32_t first_sw;        // first switch of the level-l0 block (within the permutation)
+    uint32_t x0;              // offset of the chunk inside that block
+    int m0;                   // log2 of the level-l0 block size
+    int n;
+};
+
+__device__ __forceinline__ uint32_t cross_bit(const Geometry &g, int stage, uint32_t u, int i) {
+    const uint32_t sw = g.first_sw + (rev_bits(u & ((1u << i) - 1u), i) << (g.m0 - 1 - i)) +
+                        (g.x0 >> (i + 1)) + (u >> (i + 1));
+    return (__ldg(g.bits_p + size_t(stage) * g.stage_w + (sw >> 5)) >> (sw & 31u)) & 1u;
+}
+
+// Stages on slot bits [ilo, ilo + r) of a chunk of 2^cbits slots.  Ascending
+// (input side: stage number l0 + i) or descending (output side: 2n-2-(l0+i)).
+template <typename E, bool OUT>
+__device__ __forceinline__ void run_round(E *sm, const Geometry &g, int l0, int cbits, int ilo, int r) {
+    const uint32_t groups = 1u << (cbits - r);
+    for (uint32_t gi = threadIdx.x; gi < groups; gi += blockDim.x) {
+        const uint32_t u0 = ((gi >> ilo) << (ilo + r)) | (gi & ((1u << ilo) - 1u));
+        E e[1 << kRound];
+#pragma unroll
+        for (int q = 0; q < (1 << kRound); ++q)
+            if (q < (1 << r)) e[q] = sm[phys(u0 | (uint32_t(q) << ilo))];
+#pragma unroll
+        for (int jj = 0; jj < kRound; ++jj) {
+            const int j = OUT ? (kRound - 1 - jj) : jj;     // descending on the output side
+            if (j < r) {
+                const int i = ilo + j;
+                const int stage = OUT ? (2 * g.n - 2 - (l0 + i)) : (l0 + i);
+#pragma unroll
+                for (int q = 0; q < (1 << kRound); ++q) {
+                    if (q < (1 << r) && !(q & (1 << j))) {
+                        const uint32_t c = cross_bit(g, stage, u0 | (uint32_t(q) << ilo), i);
+                        const E a = e[q], b = e[q | (1 << j)];
+                        e[q] = c ? b : a;
+                        e[q | (1 << j)] = c ? a : b;
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int q = 0; q < (1 << kRound); ++q)
+            if (q < (1 << r)) sm[phys(u0 | (uint32_t(q) << ilo))] = e[q];
+    }
+}
+
+__device__ __forceinline__ Geometry geometry(const uint32_t *bits, size_t flat, int n, int m0) {
+    Geometry g;
+    const size_t N = size_t(1) << n;
+    g.stage_w = n >= 6 ? (1u << (n - 6)) : 1u;
+    g.bits_p = bits + (flat >> n) * size_t(2 * n - 1) * g.stage_w;
+    const uint32_t local = uint32_t(flat & (N - 1));
+    const uint32_t block = local & ~((1u << m0) - 1u);
+    g.first_sw = block >> 1;
+    g.x0 = local - block;
+    g.m0 = m0;
+    g.n = n;
+    return g;
+}
+
+// Inner kernel: all 2b-1 stages of one block of 2^b elements of level n-b.
+template <typename E>
+__global__ void __launch_bounds__(kApplyThreads)
+k_apply_inner(const uint32_t *__restrict__ bits, const E *__restrict__ x, E *__restrict__ y, int n, int b) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    E *sm = reinterpret_cast<E *>(smem_raw);
+    const size_t flat0 = size_t(blockIdx.x) << b;
+    const Geometry g = geometry(bits, flat0, n, b);
+    const int l0 = n - b;
+    const uint32_t B = 1u << b;
+    for (uint32_t u = threadIdx.x; u < B; u += blockDim.x) sm[phys(u)] = x[flat0 + u];
+    __syncthreads();
+    for (int ilo = 0; ilo < b; ilo += kRound) {                     // input side and middle
+        run_round<E, false>(sm, g, l0, b, ilo, min(kRound, b - ilo));
+        __syncthreads();
+    }
+    for (int ihi = b - 2; ihi >= 0; ihi -= kRound) {                // output side
+        const int r = min(kRound, ihi + 1);
+        run_round<E, true>(sm, g, l0, b, ihi - r + 1, r);
+        __syncthreads();
+    }
+    for (uint32_t u = threadIdx.x; u < B; u += blockDim.x) y[flat0 + u] = sm[phys(u)];
+}
+
+// Outer kernel, input side (OUT = false): stages l0 .. l0+k-1 on a contiguous
+// chunk; output side (OUT = true): stages 2n-2-(l0+k-1) .. 2n-2-l0, chunk
+// gathered from its 2^k runs and written contiguously.
+template <typename E, bool OUT>
+__global__ void __launch_bounds__(kApplyThreads)
+k_apply_outer(const uint32_t *__restrict__ bits, const E *__restrict__ x, E *__restrict__ y, int n,
+              int l0, int k) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    E *sm = reinterpret_cast<E *>(smem_raw);
+    const size_t flat0 = size_t(blockIdx.x) << kChunkLog2;
+    const int m0 = n - l0;
+    const Geometry g = geometry(bits, flat0, n, m0);
+    const int tbits = kChunkLog2 - k;                               // log2 of the run length T
+    const uint32_t tmask = (1u << tbits) - 1u;
+    // flat start of the level-l0 block, and the first position of the runs inside it
+    const size_t block0 = flat0 - g.x0;
+    const uint32_t y0 = g.x0 >> k;
+    if (!OUT) {
+        for (uint32_t u = threadIdx.x; u < uint32_t(kChunk); u += blockDim.x) sm[phys(u)] = x[flat0 + u];
+    } else {
+        for (uint32_t idx = threadIdx.x; idx < uint32_t(kChunk); idx += blockDim.x) {
+            const uint32_t c = idx >> tbits, yy = idx & tmask;
+            sm[phys((yy << k) | c)] = x[block0 + (size_t(rev_bits(c, k)) << (m0 - k)) + y0 + yy];
+        }
+    }
+    __syncthreads();
+    if (!OUT) {
+        for (int ilo = 0; ilo < k; ilo += kRound) {
+            run_round<E, false>(sm, g, l0, kChunkLog2, ilo, min(kRound, k - ilo));
+            __syncthreads();
+        }
+        for (uint32_t idx = threadIdx.x; idx < uint32_t(kChunk); idx += blockDim.x) {
+            const uint32_t c = idx >> tbits, yy = idx & tmask;
+            y[block0 + (size_t(rev_bits(c, k)) << (m0 - k)) + y0 + yy] = sm[phys((yy << k) | c)];
+        }
+    } else {
+        for (int ihi = k - 1; ihi >= 0; ihi -= kRound) {
+            const int r = min(kRound, ihi + 1);
+            run_round<E, true>(sm, g, l0, kChunkLog2, ihi - r + 1, r);
+            __syncthreads();
+        }
+        for (uint32_t u = threadIdx.x; u < uint32_t(kChunk); u += blockDim.x) y[flat0 + u] = sm[phys(u)];
+    }
+}
+
+template <typename K>
+int opt_in_smem(K kernel, size_t bytes) {
+    if (bytes > 48 * 1024)
+        BENES_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(bytes)));
+    return BENES_OK;
+}
+
+template <typename E>
+int apply_fused_typed(const uint32_t *bits, const E *in, E *out, E *scratch, int n, size_t batch,
+                      cudaStream_t s) {
+    const size_t total = batch << n;
+    const size_t smem = size_t(kSmemElems) * sizeof(E);
+    static bool configured = false;
+    if (!configured) {
+        int rc;
+        if ((rc = opt_in_smem(k_apply_inner<E>, smem))) return rc;
+        if ((rc = opt_in_smem(k_apply_outer<E, false>, smem))) return rc;
+        if ((rc = opt_in_smem(k_apply_outer<E, true>, smem))) return rc;
+        configured = true;
+    }
+    const int b = n < kChunkLog2 ? n : kChunkLog2;
+    const int outer = n - b;                       // levels handled by the outer kernels, per side
+    const int per_side = (outer + 6) / 7;          // passes per side, at most 7 stages each
+    const int passes = 2 * per_side + 1;
+    // split `outer` levels evenly over the passes of a side
+    int ks[8] = {0};
+    for (int i = 0; i < per_side; ++i) ks[i] = outer / per_side + (i < outer % per_side ? 1 : 0);
+
+    // ping-pong between `out` and the scratch buffer so that the last pass lands in `out`
+    const E *src = in;
+    int pass = 0;
+    auto next_dst = [&]() { ++pass; return ((passes - pass) % 2 == 0) ? out : scratch; };
+    const unsigned chunks = unsigned(total >> kChunkLog2);
+    int l0 = 0;
+    for (int i = 0; i < per_side; ++i) {
+        E *dst = next_dst();
+        k_apply_outer<E, false><<<chunks, kApplyThreads, smem, s>>>(bits, src, dst, n, l0, ks[i]);
+        int rc = launch_status();
+        if (rc) return rc;
+        src = dst;
+        l0 += ks[i];
+    }
+    {
+        E *dst = next_dst();
+        const unsigned blocks = unsigned(total >> b);
+        const unsigned threads = (1u << b) >> kRound < 32u ? 32u : (1u << b) >> kRound;
+        k_apply_inner<E><<<blocks, threads, smem, s>>>(bits, src, dst, n, b);
+        int rc = launch_status();
+        if (rc) return rc;
+        src = dst;
+    }
+    for (int i = per_side - 1; i >= 0; --i) {
+        E *dst = next_dst();
+        l0 -= ks[i];
+        k_apply_outer<E, true><<<chunks, kApplyThreads, smem, s>>>(bits, src, dst, n, l0, ks[i]);
+        int rc = launch_status();
+        if (rc) return rc;
+        src = dst;
+    }
+    return BENES_OK;
+}
+
+}  // namespace
+
+int apply_fused_passes(int log2n) {
+    const int b = log2n < kChunkLog2 ? log2n : kChunkLog2;
+    return 2 * ((log2n - b + 6) / 7) + 1;
+}
+
+int launch_apply_fused(const uint32_t *bits, const void *in, void *out, void *scratch, int elem_bytes,
+                       int log2n, size_t batch, cudaStream_t s) {
+    if (elem_bytes == 4)
+        return apply_fused_typed<uint32_t>(bits, static_cast<const uint32_t *>(in),
+                                           static_cast<uint32_t *>(out), static_cast<uint32_t *>(scratch),
+                                           log2n, batch, s);
+    if (elem_bytes == 8)
+        return apply_fused_typed<unsigned long long>(bits, static_cast<const unsigned long long *>(in),
+                                                     static_cast<unsigned long long *>(out),
+                                                     static_cast<unsigned long long *>(scratch), log2n,
+                                                     batch, s);
+    return BENES_ERR_BADARG;
+}
+
+}  // namespace benes

@@ -26,6 +26,7 @@ std::mutex g_mu;
 // jumping over all outputs; 2..8: one ruler switch per 2^kappa switches.
 int g_kappa = 4;
 int g_walk_cap = 1 << 14;
+int g_apply_fused = 1;
 constexpr int kMaxLevels = 32;
 
 inline size_t align_up(size_t v) { return (v + kAlign - 1) & ~(kAlign - 1); }
@@ -239,7 +240,12 @@ int benes_apply_ex(const uint32_t *switch_bits, const void *in, void *out, int e
         int rc = get_workspace(apply_ws_bytes(elem_bytes, n, size_t(batch)), &ws);
         if (rc) return rc;
     }
-    // ping-pong between `out` and the scratch buffer so that the last stage lands in `out`
+    if (g_apply_fused) {
+        ProfileScope ps(kApplyFused, s);
+        return launch_apply_fused(switch_bits, in, out, ws, elem_bytes, n, size_t(batch), s);
+    }
+    // one stage per launch: ping-pong between `out` and the scratch buffer so
+    // that the last stage lands in `out`
     const void *src = in;
     ProfileScope ps(kApply, s);
     for (int st = 0; st < stages; ++st) {
@@ -332,6 +338,10 @@ int benes_set_option(int key, int value) {
             if (value < 1 || value > (1 << 24)) return BENES_ERR_BADARG;
             g_walk_cap = value;
             return BENES_OK;
+        case BENES_OPT_APPLY_FUSED:
+            if (value != 0 && value != 1) return BENES_ERR_BADARG;
+            g_apply_fused = value;
+            return BENES_OK;
         default: return BENES_ERR_BADARG;
     }
 }
@@ -341,6 +351,7 @@ int benes_get_option(int key) {
     switch (key) {
         case BENES_OPT_SAMPLE_LOG2K: return g_kappa;
         case BENES_OPT_WALK_CAP: return g_walk_cap;
+        case BENES_OPT_APPLY_FUSED: return g_apply_fused;
         default: return BENES_ERR_BADARG;
     }
 }

@@ -119,6 +119,12 @@ int launch_fused(const void *P, int records, size_t total, int log2m, uint32_t *
 int launch_apply_stage(const uint32_t *bits, const void *x, void *y, int elem_bytes, int stage,
                        int log2n, size_t batch, cudaStream_t s);
 
+// ---- payload apply, several stages per pass (apply_fused.cu) -----------------
+// `scratch` (batch * N elements) is needed when apply_fused_passes(log2n) > 1.
+int apply_fused_passes(int log2n);
+int launch_apply_fused(const uint32_t *bits, const void *in, void *out, void *scratch, int elem_bytes,
+                       int log2n, size_t batch, cudaStream_t s);
+
 // ---- validation (route_levels.cu) -------------------------------------------
 int launch_validate(const uint32_t *perm, size_t total, int log2n, uint32_t *seen_words,
                     uint32_t *flag, cudaStream_t s);

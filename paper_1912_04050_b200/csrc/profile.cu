@@ -94,6 +94,20 @@ int benes_profile_read(int kind, unsigned long long *launches, double *milliseco
     return BENES_OK;
 }
 
+int benes_profile_span(int index, int *kind, unsigned long long *launches, double *milliseconds) {
+    if (index < 0 || !kind || !launches || !milliseconds) return BENES_ERR_BADARG;
+    std::lock_guard<std::mutex> lk(g_pmu);
+    if (index >= int(g_spans.size())) return BENES_ERR_BADARG;
+    Span &sp = g_spans[index];
+    float t = 0.f;
+    BENES_CUDA_TRY(cudaEventSynchronize(sp.stop));
+    BENES_CUDA_TRY(cudaEventElapsedTime(&t, sp.start, sp.stop));
+    *kind = sp.kind;
+    *launches = sp.launches;
+    *milliseconds = t;
+    return BENES_OK;
+}
+
 const char *benes_profile_kind_name(int kind) {
     return (kind >= 0 && kind < BENES_PROFILE_KINDS) ? kNames[kind] : "?";
 }

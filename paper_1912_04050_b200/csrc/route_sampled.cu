@@ -36,12 +36,13 @@
 #include "common.cuh"
 
 namespace benes {
+
+
 namespace {
 
 constexpr int kThreads = 256;
 constexpr int kSMs = 148;
 constexpr int kListThreads = 1024;
-constexpr int kListPer = (1 << kListSmemLog2) / kListThreads;   // words per thread, at most
 
 __device__ __forceinline__ uint32_t ruler_slot(uint32_t group, uint32_t salt, uint32_t kmask) {
     uint32_t h = group * 0x9E3779B1u + salt;
@@ -182,43 +183,56 @@ k_list_resolve(unsigned long long *__restrict__ W, uint32_t *__restrict__ owner,
 
 // Step 4, the end of the recursion: one CTA labels one block's list of
 // 2^log2b words in shared memory by synchronous pointer jumping (new words are
-// held in registers across the barrier).  A cycle has at most 2^log2b words
-// (a list sampled from a list need not split evenly between a cycle and its
-// mirror image), hence log2b passes.
+// held in registers across the barrier; PER words per thread, blockDim =
+// 2^log2b / PER).  A cycle has at most 2^log2b words (a list sampled from a
+// list need not split evenly between a cycle and its mirror image), hence
+// log2b passes.
+template <int PER>
 __global__ void __launch_bounds__(kListThreads)
 k_list_label(unsigned long long *__restrict__ W, int log2b) {
     extern __shared__ unsigned long long sm[];
     const uint32_t B = 1u << log2b, bmask = B - 1u;
     const size_t base = size_t(blockIdx.x) << log2b;
     const uint32_t T = blockDim.x, tid = threadIdx.x;
-    for (uint32_t e = tid; e < B; e += T) {
+#pragma unroll
+    for (int i = 0; i < PER; ++i) {
+        const uint32_t e = tid + uint32_t(i) * T;
         unsigned long long w = __ldcs(W + base + e);
         sm[e] = make_word(uint32_t(w) & bmask, uint32_t(w >> 32));
     }
     __syncthreads();
-    unsigned long long v[kListPer];
+    unsigned long long v[PER];
     for (int pass = 0; pass < log2b; ++pass) {
 #pragma unroll
-        for (int i = 0; i < kListPer; ++i) {
-            const uint32_t e = tid + uint32_t(i) * T;
-            if (e < B) {
-                const unsigned long long w = sm[e];
-                const unsigned long long t = sm[uint32_t(w)];
-                v[i] = make_word(uint32_t(t), min(uint32_t(w >> 32), uint32_t(t >> 32)));
-            }
+        for (int i = 0; i < PER; ++i) {
+            const unsigned long long w = sm[tid + uint32_t(i) * T];
+            const unsigned long long t = sm[uint32_t(w)];
+            v[i] = make_word(uint32_t(t), min(uint32_t(w >> 32), uint32_t(t >> 32)));
         }
         __syncthreads();
 #pragma unroll
-        for (int i = 0; i < kListPer; ++i) {
-            const uint32_t e = tid + uint32_t(i) * T;
-            if (e < B) sm[e] = v[i];
-        }
+        for (int i = 0; i < PER; ++i) sm[tid + uint32_t(i) * T] = v[i];
         __syncthreads();
     }
-    for (uint32_t e = tid; e < B; e += T) {
+#pragma unroll
+    for (int i = 0; i < PER; ++i) {
+        const uint32_t e = tid + uint32_t(i) * T;
         const unsigned long long w = sm[e];
         W[base + e] = make_word(uint32_t(base) + uint32_t(w), uint32_t(w >> 32));
     }
+}
+
+template <int PER>
+int launch_list_label(unsigned long long *W, uint32_t count, int beta, cudaStream_t s) {
+    static bool configured = false;
+    const size_t smem = (size_t(1) << beta) * 8;
+    if (!configured) {
+        BENES_CUDA_TRY(cudaFuncSetAttribute(k_list_label<PER>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            (1 << kListSmemLog2) * 8));
+        configured = true;
+    }
+    k_list_label<PER><<<count >> beta, (1u << beta) / PER, smem, s>>>(W, beta);
+    return launch_status();
 }
 
 // Step 5 + output side of the level's switches.
@@ -342,17 +356,11 @@ int sampled_label(uint4 *S, const uint32_t *Q, const SampledScratch &sc, size_t 
     }
     {
         ProfileScope ps(kListLabel, s);
-        static bool configured = false;
-        if (!configured) {
-            BENES_CUDA_TRY(cudaFuncSetAttribute(k_list_label, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                (1 << kListSmemLog2) * 8));
-            configured = true;
-        }
-        if (beta > kListSmemLog2) return BENES_ERR_BADARG;
-        const uint32_t B = 1u << beta;
-        const unsigned threads = B < unsigned(kListThreads) ? (B < 32u ? 32u : B) : unsigned(kListThreads);
-        k_list_label<<<count >> beta, threads, size_t(B) * 8, s>>>(sc.list[depth], beta);
-        int rc = launch_status();
+        if (beta > kListSmemLog2 || beta < 5) return BENES_ERR_BADARG;
+        // 4 words per thread up to 2^12 words, then 1024 threads
+        int rc = beta <= 12 ? launch_list_label<4>(sc.list[depth], count, beta, s)
+               : beta == 13 ? launch_list_label<8>(sc.list[depth], count, beta, s)
+                            : launch_list_label<16>(sc.list[depth], count, beta, s);
         if (rc) return rc;
     }
     for (int d = depth - 1; d >= 0; --d) {

@@ -85,6 +85,15 @@ def labelling_options():
     binding.benes_set_option(binding.OPT_WALK_CAP, c0)
 
 
+@pytest.fixture(params=[1, 0], ids=["fused", "per_stage"])
+def apply_mode(request):
+    """Both payload-apply paths: several stages per pass, and one stage per pass."""
+    a0 = binding.benes_get_option(binding.OPT_APPLY_FUSED)
+    binding.benes_set_option(binding.OPT_APPLY_FUSED, request.param)
+    yield request.param
+    binding.benes_set_option(binding.OPT_APPLY_FUSED, a0)
+
+
 @pytest.mark.parametrize("kappa", [0, 2, 3, 5, 8])
 def test_route_every_ruler_spacing(kappa, labelling_options):
     """0 = pointer jumping over all outputs; otherwise one ruler per 2^kappa switches."""
@@ -112,12 +121,12 @@ def test_route_walks_that_give_up_fall_back_to_full_pointer_jumping(cap, labelli
 
 
 # ---- apply ------------------------------------------------------------------
-@pytest.mark.parametrize("n", [1, 2, 3, 5, 6, 7, 10, 13, 16])
+@pytest.mark.parametrize("n", [1, 2, 3, 4, 5, 6, 7, 10, 12, 13, 14, 16, 19, 21])
 @pytest.mark.parametrize("dtype", [np.uint32, np.uint64])
-def test_apply_random_settings(n, dtype):
+def test_apply_random_settings(n, dtype, apply_mode):
     """Arbitrary switch settings (not produced by route): checks wiring and layout alone."""
     rng = np.random.default_rng(n)
-    batch = 3
+    batch = 3 if n < 19 else 1
     W = max(1, (1 << n) // 64)
     bits = rng.integers(0, 2 ** 32, size=(batch, 2 * n - 1, W), dtype=np.uint64).astype(np.uint32)
     if n < 6:
