@@ -25,7 +25,8 @@
 // written at the end.  The output side reads the same relation backwards.
 //
 // A thread holds 8 slots (3 slot bits) in registers and runs 3 stages between
-// two barriers.
+// two barriers; the switch words of all stages of the pass are staged in
+// shared memory first.
 #include "common.cuh"
 
 namespace benes {
@@ -36,8 +37,12 @@ constexpr int kChunk = 1 << kChunkLog2;
 constexpr int kRound = 3;                    // stages between barriers
 constexpr int kApplyThreads = kChunk >> kRound;
 
-__device__ __forceinline__ uint32_t phys(uint32_t u) { return u + (u >> 5); }
-constexpr int kSmemElems = kChunk + (kChunk >> 5);
+// Slot u lives at shared-memory index phys(u): an XOR swizzle of the low bits,
+// chosen so that every access pattern of the kernels (consecutive slots; the
+// 8-slot groups of each round; columns of the 2^k x T transposition of the
+// outer kernels) spreads a warp over all banks.
+__device__ __forceinline__ uint32_t phys(uint32_t u) { return u ^ ((u >> 3) & 31u) ^ ((u >> 7) & 31u); }
+constexpr int kSmemElems = kChunk;
 
 __device__ __forceinline__ uint32_t rev_bits(uint32_t v, int i) {
     return i ? (__brev(v) >> (32 - i)) : 0u;
@@ -52,44 +57,86 @@ struct Geometry {
     int n;
 };
 
-__device__ __forceinline__ uint32_t cross_bit(const Geometry &g, int stage, uint32_t u, int i) {
-    const uint32_t sw = g.first_sw + (rev_bits(u & ((1u << i) - 1u), i) << (g.m0 - 1 - i)) +
-                        (g.x0 >> (i + 1)) + (u >> (i + 1));
-    return (__ldg(g.bits_p + size_t(stage) * g.stage_w + (sw >> 5)) >> (sw & 31u)) & 1u;
+// The switch words a CTA needs are copied to shared memory first: kBitWords
+// words per stage, the stage's runs (one run per path through the earlier
+// stages of the pass) one after the other.  Stage l0+i of a chunk of 2^cbits
+// slots has 2^i runs of 2^(cbits-1-i) switches; run c starts at switch
+//     first_sw + (c << (m0-1-i)) + (x0 >> (i+1)).
+// In the inner kernel (x0 = 0, m0 = cbits) the runs of a stage are contiguous,
+// so the stage is one piece of 2^(cbits-1) bits.
+constexpr int kBitWords = kChunk / 64;
+
+template <bool OUT>
+__device__ __forceinline__ void stage_bits_to_smem(uint32_t *sb, const Geometry &g, int l0, int cbits,
+                                                   int i_count, int slot0) {
+    const int wbits = cbits > 6 ? cbits - 6 : 0;          // log2(words per stage), at least one word
+    for (uint32_t idx = threadIdx.x; idx < uint32_t(i_count) << wbits; idx += blockDim.x) {
+        const int i = int(idx >> wbits);
+        const uint32_t r = idx & ((1u << wbits) - 1u);
+        const int rw = wbits - i;                         // log2(words per run); < 0: runs inside a word
+        const int stage = OUT ? (2 * g.n - 2 - (l0 + i)) : (l0 + i);
+        const uint32_t *src = g.bits_p + size_t(stage) * g.stage_w;
+        uint32_t word;
+        if (rw >= 0) {
+            const uint32_t c = r >> rw, w = r & ((1u << rw) - 1u);
+            const uint32_t sw = g.first_sw + (c << (g.m0 - 1 - i)) + (g.x0 >> (i + 1));
+            word = __ldg(src + (sw >> 5) + w);
+        } else {
+            word = __ldg(src + (g.first_sw >> 5) + r);    // inner kernel only: contiguous
+        }
+        sb[(slot0 + i) * kBitWords + r] = word;
+    }
 }
 
-// Stages on slot bits [ilo, ilo + r) of a chunk of 2^cbits slots.  Ascending
-// (input side: stage number l0 + i) or descending (output side: 2n-2-(l0+i)).
-template <typename E, bool OUT>
-__device__ __forceinline__ void run_round(E *sm, const Geometry &g, int l0, int cbits, int ilo, int r) {
-    const uint32_t groups = 1u << (cbits - r);
+// R stages on slot bits [ilo, ilo + R) of a chunk of 2^cbits slots: ascending
+// on the input side, descending on the output side.  sb + (slot_of_i0 + i) *
+// kBitWords = words of the stage on slot bit i.  A thread holds the 2^R slots
+// u0 | (q << ilo).  The switch of the pair (q, q | 1 << j) of stage i = ilo+j
+// is bit  (rev_i(low i bits of the slot) << (cbits-1-i)) + (slot >> (i+1))  of
+// the stage: the bits of q below j move the run, the bits above j are
+// neighbouring switches of one word.
+template <typename E, bool OUT, int R>
+__device__ __forceinline__ void run_round(E *sm, const uint32_t *sb, int slot_of_i0, int cbits, int ilo) {
+    const uint32_t groups = 1u << (cbits - R);
     for (uint32_t gi = threadIdx.x; gi < groups; gi += blockDim.x) {
-        const uint32_t u0 = ((gi >> ilo) << (ilo + r)) | (gi & ((1u << ilo) - 1u));
-        E e[1 << kRound];
+        const uint32_t u0 = ((gi >> ilo) << (ilo + R)) | (gi & ((1u << ilo) - 1u));
+        E e[1 << R];
 #pragma unroll
-        for (int q = 0; q < (1 << kRound); ++q)
-            if (q < (1 << r)) e[q] = sm[phys(u0 | (uint32_t(q) << ilo))];
+        for (int q = 0; q < (1 << R); ++q) e[q] = sm[phys(u0 | (uint32_t(q) << ilo))];
 #pragma unroll
-        for (int jj = 0; jj < kRound; ++jj) {
-            const int j = OUT ? (kRound - 1 - jj) : jj;     // descending on the output side
-            if (j < r) {
-                const int i = ilo + j;
-                const int stage = OUT ? (2 * g.n - 2 - (l0 + i)) : (l0 + i);
+        for (int jj = 0; jj < R; ++jj) {
+            const int j = OUT ? (R - 1 - jj) : jj;
+            const int i = ilo + j, sh = cbits - 1 - i;
+            const uint32_t idx0 = (rev_bits(u0 & ((1u << i) - 1u), i) << sh) + (u0 >> (i + 1));
+            const uint32_t *words = sb + (slot_of_i0 + i) * kBitWords;
 #pragma unroll
-                for (int q = 0; q < (1 << kRound); ++q) {
-                    if (q < (1 << r) && !(q & (1 << j))) {
-                        const uint32_t c = cross_bit(g, stage, u0 | (uint32_t(q) << ilo), i);
-                        const E a = e[q], b = e[q | (1 << j)];
-                        e[q] = c ? b : a;
-                        e[q | (1 << j)] = c ? a : b;
-                    }
+            for (int lo = 0; lo < (1 << j); ++lo) {
+                uint32_t crev = 0;                        // lo with its j bits reversed
+#pragma unroll
+                for (int t = 0; t < j; ++t) crev |= ((uint32_t(lo) >> t) & 1u) << (j - 1 - t);
+                const uint32_t idx = idx0 + (crev << sh);
+                const uint32_t w = words[idx >> 5] >> (idx & 31u);
+#pragma unroll
+                for (int hi = 0; hi < (1 << (R - 1 - j)); ++hi) {
+                    const int q = lo | (hi << (j + 1));
+                    const bool cross = (w >> hi) & 1u;
+                    const E a = e[q], b = e[q | (1 << j)];
+                    e[q] = cross ? b : a;
+                    e[q | (1 << j)] = cross ? a : b;
                 }
             }
         }
 #pragma unroll
-        for (int q = 0; q < (1 << kRound); ++q)
-            if (q < (1 << r)) sm[phys(u0 | (uint32_t(q) << ilo))] = e[q];
+        for (int q = 0; q < (1 << R); ++q) sm[phys(u0 | (uint32_t(q) << ilo))] = e[q];
     }
+}
+
+template <typename E, bool OUT>
+__device__ __forceinline__ void run_round_r(E *sm, const uint32_t *sb, int slot_of_i0, int cbits, int ilo,
+                                            int r) {
+    if (r == 3) run_round<E, OUT, 3>(sm, sb, slot_of_i0, cbits, ilo);
+    else if (r == 2) run_round<E, OUT, 2>(sm, sb, slot_of_i0, cbits, ilo);
+    else run_round<E, OUT, 1>(sm, sb, slot_of_i0, cbits, ilo);
 }
 
 __device__ __forceinline__ Geometry geometry(const uint32_t *bits, size_t flat, int n, int m0) {
@@ -116,15 +163,20 @@ k_apply_inner(const uint32_t *__restrict__ bits, const E *__restrict__ x, E *__r
     const Geometry g = geometry(bits, flat0, n, b);
     const int l0 = n - b;
     const uint32_t B = 1u << b;
+    // words of the b input-side + middle stages in slots 0..b-1, of the b-1
+    // output-side stages in slots b..2b-2 (slot b+i for slot bit i)
+    uint32_t *sb = reinterpret_cast<uint32_t *>(sm + kSmemElems);
+    stage_bits_to_smem<false>(sb, g, l0, b, b, 0);
+    stage_bits_to_smem<true>(sb, g, l0, b, b - 1, b);
     for (uint32_t u = threadIdx.x; u < B; u += blockDim.x) sm[phys(u)] = x[flat0 + u];
     __syncthreads();
     for (int ilo = 0; ilo < b; ilo += kRound) {                     // input side and middle
-        run_round<E, false>(sm, g, l0, b, ilo, min(kRound, b - ilo));
+        run_round_r<E, false>(sm, sb, 0, b, ilo, min(kRound, b - ilo));
         __syncthreads();
     }
     for (int ihi = b - 2; ihi >= 0; ihi -= kRound) {                // output side
         const int r = min(kRound, ihi + 1);
-        run_round<E, true>(sm, g, l0, b, ihi - r + 1, r);
+        run_round_r<E, true>(sm, sb, b, b, ihi - r + 1, r);
         __syncthreads();
     }
     for (uint32_t u = threadIdx.x; u < B; u += blockDim.x) y[flat0 + u] = sm[phys(u)];
@@ -147,6 +199,8 @@ k_apply_outer(const uint32_t *__restrict__ bits, const E *__restrict__ x, E *__r
     // flat start of the level-l0 block, and the first position of the runs inside it
     const size_t block0 = flat0 - g.x0;
     const uint32_t y0 = g.x0 >> k;
+    uint32_t *sb = reinterpret_cast<uint32_t *>(sm + kSmemElems);
+    stage_bits_to_smem<OUT>(sb, g, l0, kChunkLog2, k, 0);
     if (!OUT) {
         for (uint32_t u = threadIdx.x; u < uint32_t(kChunk); u += blockDim.x) sm[phys(u)] = x[flat0 + u];
     } else {
@@ -158,7 +212,7 @@ k_apply_outer(const uint32_t *__restrict__ bits, const E *__restrict__ x, E *__r
     __syncthreads();
     if (!OUT) {
         for (int ilo = 0; ilo < k; ilo += kRound) {
-            run_round<E, false>(sm, g, l0, kChunkLog2, ilo, min(kRound, k - ilo));
+            run_round_r<E, false>(sm, sb, 0, kChunkLog2, ilo, min(kRound, k - ilo));
             __syncthreads();
         }
         for (uint32_t idx = threadIdx.x; idx < uint32_t(kChunk); idx += blockDim.x) {
@@ -168,7 +222,7 @@ k_apply_outer(const uint32_t *__restrict__ bits, const E *__restrict__ x, E *__r
     } else {
         for (int ihi = k - 1; ihi >= 0; ihi -= kRound) {
             const int r = min(kRound, ihi + 1);
-            run_round<E, true>(sm, g, l0, kChunkLog2, ihi - r + 1, r);
+            run_round_r<E, true>(sm, sb, 0, kChunkLog2, ihi - r + 1, r);
             __syncthreads();
         }
         for (uint32_t u = threadIdx.x; u < uint32_t(kChunk); u += blockDim.x) y[flat0 + u] = sm[phys(u)];
@@ -186,7 +240,8 @@ template <typename E>
 int apply_fused_typed(const uint32_t *bits, const E *in, E *out, E *scratch, int n, size_t batch,
                       cudaStream_t s) {
     const size_t total = batch << n;
-    const size_t smem = size_t(kSmemElems) * sizeof(E);
+    // payload slots + the switch words of up to 2*13-1 stages
+    const size_t smem = size_t(kSmemElems) * sizeof(E) + size_t(2 * kChunkLog2 - 1) * kBitWords * 4;
     static bool configured = false;
     if (!configured) {
         int rc;
