@@ -35,7 +35,7 @@ namespace {
 constexpr int kChunkLog2 = 13;               // elements per CTA
 constexpr int kChunk = 1 << kChunkLog2;
 constexpr int kRound = 3;                    // stages between barriers
-constexpr int kApplyThreads = kChunk >> kRound;
+constexpr int kApplyThreads = 512;           // two 8-slot groups per thread and round, two CTAs per SM
 
 // Slot u lives at shared-memory index phys(u): an XOR swizzle of the low bits,
 // chosen so that every access pattern of the kernels (consecutive slots; the
@@ -98,11 +98,16 @@ __device__ __forceinline__ void stage_bits_to_smem(uint32_t *sb, const Geometry 
 template <typename E, bool OUT, int R>
 __device__ __forceinline__ void run_round(E *sm, const uint32_t *sb, int slot_of_i0, int cbits, int ilo) {
     const uint32_t groups = 1u << (cbits - R);
+    // phys is linear over XOR and the slots of a group differ from u0 in bits u0 lacks
+    uint32_t dq[1 << R];
+#pragma unroll
+    for (int q = 0; q < (1 << R); ++q) dq[q] = phys(uint32_t(q) << ilo);
     for (uint32_t gi = threadIdx.x; gi < groups; gi += blockDim.x) {
         const uint32_t u0 = ((gi >> ilo) << (ilo + R)) | (gi & ((1u << ilo) - 1u));
+        const uint32_t p0 = phys(u0);
         E e[1 << R];
 #pragma unroll
-        for (int q = 0; q < (1 << R); ++q) e[q] = sm[phys(u0 | (uint32_t(q) << ilo))];
+        for (int q = 0; q < (1 << R); ++q) e[q] = sm[p0 ^ dq[q]];
 #pragma unroll
         for (int jj = 0; jj < R; ++jj) {
             const int j = OUT ? (R - 1 - jj) : jj;
@@ -127,7 +132,7 @@ __device__ __forceinline__ void run_round(E *sm, const uint32_t *sb, int slot_of
             }
         }
 #pragma unroll
-        for (int q = 0; q < (1 << R); ++q) sm[phys(u0 | (uint32_t(q) << ilo))] = e[q];
+        for (int q = 0; q < (1 << R); ++q) sm[p0 ^ dq[q]] = e[q];
     }
 }
 
@@ -155,7 +160,7 @@ __device__ __forceinline__ Geometry geometry(const uint32_t *bits, size_t flat, 
 
 // Inner kernel: all 2b-1 stages of one block of 2^b elements of level n-b.
 template <typename E>
-__global__ void __launch_bounds__(kApplyThreads)
+__global__ void __launch_bounds__(kApplyThreads, 2)
 k_apply_inner(const uint32_t *__restrict__ bits, const E *__restrict__ x, E *__restrict__ y, int n, int b) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     E *sm = reinterpret_cast<E *>(smem_raw);
@@ -186,7 +191,7 @@ k_apply_inner(const uint32_t *__restrict__ bits, const E *__restrict__ x, E *__r
 // chunk; output side (OUT = true): stages 2n-2-(l0+k-1) .. 2n-2-l0, chunk
 // gathered from its 2^k runs and written contiguously.
 template <typename E, bool OUT>
-__global__ void __launch_bounds__(kApplyThreads)
+__global__ void __launch_bounds__(kApplyThreads, 2)
 k_apply_outer(const uint32_t *__restrict__ bits, const E *__restrict__ x, E *__restrict__ y, int n,
               int l0, int k) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -233,6 +238,9 @@ template <typename K>
 int opt_in_smem(K kernel, size_t bytes) {
     if (bytes > 48 * 1024)
         BENES_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(bytes)));
+    // room for two CTAs per SM
+    BENES_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                        cudaSharedmemCarveoutMaxShared));
     return BENES_OK;
 }
 
@@ -275,7 +283,8 @@ int apply_fused_typed(const uint32_t *bits, const E *in, E *out, E *scratch, int
     {
         E *dst = next_dst();
         const unsigned blocks = unsigned(total >> b);
-        const unsigned threads = (1u << b) >> kRound < 32u ? 32u : (1u << b) >> kRound;
+        unsigned threads = (1u << b) >> kRound;
+        threads = threads < 32u ? 32u : (threads > unsigned(kApplyThreads) ? unsigned(kApplyThreads) : threads);
         k_apply_inner<E><<<blocks, threads, smem, s>>>(bits, src, dst, n, b);
         int rc = launch_status();
         if (rc) return rc;
