@@ -156,12 +156,16 @@ int benes_validate_perm(const uint32_t *perm, int log2n, int batch, benes_stream
  *   BENES_OPT_APPLY_FUSED : 1 (default) = benes_apply / benes_apply_ex run up to
  *       25 stages per pass over the payload in shared memory; 0 = one stage per
  *       pass.  Same result.
+ *   BENES_OPT_INVERSE_PARTITIONED : 1 (default) = for batch * N >= 2^22 the inverse
+ *       permutation of level 0 is formed by bucketing (destination, source)
+ *       pairs and scattering bucket by bucket; 0 = one pass of random writes.
  * benes_set_option returns BENES_OK or BENES_ERR_BADARG; benes_get_option
  * returns the value, or BENES_ERR_BADARG for an unknown key.
  */
 #define BENES_OPT_SAMPLE_LOG2K 0
 #define BENES_OPT_WALK_CAP 1
 #define BENES_OPT_APPLY_FUSED 2
+#define BENES_OPT_INVERSE_PARTITIONED 3
 int benes_set_option(int key, int value);
 int benes_get_option(int key);
 

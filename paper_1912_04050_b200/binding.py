@@ -188,6 +188,7 @@ PROFILE_KINDS = 12
 OPT_SAMPLE_LOG2K = 0
 OPT_WALK_CAP = 1
 OPT_APPLY_FUSED = 2
+OPT_INVERSE_PARTITIONED = 3
 
 
 def benes_set_option(key: int, value: int) -> None:

@@ -27,6 +27,7 @@ std::mutex g_mu;
 int g_kappa = 4;
 int g_walk_cap = 1 << 14;
 int g_apply_fused = 1;
+int g_inverse_partitioned = 1;
 constexpr int kMaxLevels = 32;
 
 inline size_t align_up(size_t v) { return (v + kAlign - 1) & ~(kAlign - 1); }
@@ -82,7 +83,8 @@ size_t route_ws_bytes(int log2n, size_t batch) {
     if (log2n <= kFusedLog2M) return 0;
     size_t T = level_chunk(log2n, batch) << log2n;
     return 2 * align_up(T * 8) + 2 * align_up(T * 4) + align_up(T * 8) +
-           align_up(sampled_scratch_bytes(T, kMinKappa)) + align_up(kMaxLevels * 4);
+           align_up(sampled_scratch_bytes(T, kMinKappa)) + align_up(kMaxLevels * 4) +
+           align_up(kInverseMaxBuckets * 4);
 }
 
 size_t apply_ws_bytes(int elem_bytes, int log2n, size_t batch) {
@@ -102,7 +104,8 @@ int route_levels(const uint32_t *perm, int n, size_t batch, uint32_t *bits, char
     Qbuf[1] = reinterpret_cast<uint32_t *>(ws + off); off += align_up(T * 4);
     unsigned long long *Wd = reinterpret_cast<unsigned long long *>(ws + off); off += align_up(T * 8);
     char *sampled = ws + off; off += align_up(sampled_scratch_bytes(T, kMinKappa));
-    uint32_t *gates = reinterpret_cast<uint32_t *>(ws + off);
+    uint32_t *gates = reinterpret_cast<uint32_t *>(ws + off); off += align_up(kMaxLevels * 4);
+    uint32_t *fill = reinterpret_cast<uint32_t *>(ws + off);
     const int kappa = g_kappa;
     const uint32_t cap = uint32_t(g_walk_cap);
     SampledScratch sc;
@@ -116,7 +119,14 @@ int route_levels(const uint32_t *perm, int n, size_t batch, uint32_t *bits, char
     BitsLayout L{bits, n, n - 6};
     {
         ProfileScope ps(kInverse, s);
-        if ((rc = launch_inverse(perm, Sbuf[0], Qbuf[0], T, n, s))) return rc;
+        // the 64-bit word array is free until the first level is labelled
+        // (the bucketed form needs whole buckets of 2^18 entries)
+        if (g_inverse_partitioned && T >= (size_t(1) << kInversePartitionMinLog2) &&
+            (T & ((size_t(1) << 18) - 1)) == 0)
+            rc = launch_inverse_partitioned(perm, Sbuf[0], Qbuf[0], Wd, fill, T, n, s);
+        else
+            rc = launch_inverse(perm, Sbuf[0], Qbuf[0], T, n, s);
+        if (rc) return rc;
     }
     int cur = 0;
     for (int level = 0; n - level > kFusedLog2M; ++level) {
@@ -128,7 +138,8 @@ int route_levels(const uint32_t *perm, int n, size_t batch, uint32_t *bits, char
         if (kappa) {
             // ruler-sampled labelling; raises `gate` if a walk had to give up
             gate = gates + level;
-            if ((rc = sampled_label(S, Q, sc, T, m, kappa, uint32_t(level), cap, L, out_stage, gate, s)))
+            if ((rc = sampled_label(S, Q, Sbuf[cur ^ 1], sc, T, m, kappa, uint32_t(level), cap, L, out_stage,
+                                    gate, s)))
                 return rc;
         }
         // pointer jumping over all outputs: the whole labelling when sampling is
@@ -139,7 +150,7 @@ int route_levels(const uint32_t *perm, int n, size_t batch, uint32_t *bits, char
         }
         {
             ProfileScope ps(kSplit, s);
-            if ((rc = launch_split(S, Q, Sbuf[cur ^ 1], Qbuf[cur ^ 1], T, m, L, level, out_stage, s)))
+            if ((rc = launch_split(S, Q, Sbuf[cur ^ 1], Qbuf[cur ^ 1], T, m, L, level, out_stage, gate, s)))
                 return rc;
         }
         cur ^= 1;
@@ -342,6 +353,10 @@ int benes_set_option(int key, int value) {
             if (value != 0 && value != 1) return BENES_ERR_BADARG;
             g_apply_fused = value;
             return BENES_OK;
+        case BENES_OPT_INVERSE_PARTITIONED:
+            if (value != 0 && value != 1) return BENES_ERR_BADARG;
+            g_inverse_partitioned = value;
+            return BENES_OK;
         default: return BENES_ERR_BADARG;
     }
 }
@@ -352,6 +367,7 @@ int benes_get_option(int key) {
         case BENES_OPT_SAMPLE_LOG2K: return g_kappa;
         case BENES_OPT_WALK_CAP: return g_walk_cap;
         case BENES_OPT_APPLY_FUSED: return g_apply_fused;
+        case BENES_OPT_INVERSE_PARTITIONED: return g_inverse_partitioned;
         default: return BENES_ERR_BADARG;
     }
 }

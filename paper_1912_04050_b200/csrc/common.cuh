@@ -83,14 +83,24 @@ __device__ __forceinline__ unsigned long long make_word(uint32_t nxt, uint32_t m
 // Level 0: S records from the caller's permutation, and Q[P[j]] = j.
 int launch_inverse(const uint32_t *perm, uint4 *S, uint32_t *Q, size_t total, int log2m,
                    cudaStream_t s);
+// The same for total >= 2^kInversePartitionMinLog2 in two streaming passes:
+// `pairs` = total x 8 bytes of scratch, `fill` = total >> 18 zero-initialised
+// counters (at most kInverseMaxBuckets).
+constexpr int kInversePartitionMinLog2 = 22;
+constexpr int kInverseMaxBuckets = 4096;
+int launch_inverse_partitioned(const uint32_t *perm, uint4 *S, uint32_t *Q, void *pairs, uint32_t *fill,
+                               size_t total, int log2m, cudaStream_t s);
 // Pointer jumping over all outputs (successor build, log2m-2 in-place passes,
 // last pass + output-side bits) in ONE cooperative launch; `gate` (may be
 // null) is a device word: the kernel returns at once while it is 0.
 int launch_full_label(const uint4 *S, const uint32_t *Q, unsigned long long *Wd, size_t total,
                       int log2m, BitsLayout L, int out_stage, const uint32_t *gate, cudaStream_t s);
-// Input-side bits + next level's records (owner reset) and inverses.
+// Input-side bits + next level's inverses; also the next level's records
+// (owner reset) if `gate` is null or *gate != 0 (otherwise the colouring kernel
+// of the sampled labelling has written them already).
 int launch_split(const uint4 *S, const uint32_t *Q, uint4 *Sn, uint32_t *Qn, size_t total,
-                 int log2m, BitsLayout L, int in_stage, int out_stage, cudaStream_t s);
+                 int log2m, BitsLayout L, int in_stage, int out_stage, const uint32_t *gate,
+                 cudaStream_t s);
 
 // ---- ruler-sampled loop labelling (route_sampled.cu) --------------------------
 struct SampledScratch {
@@ -100,10 +110,11 @@ struct SampledScratch {
 };
 size_t sampled_scratch_bytes(size_t total, int kappa);
 void sampled_scratch_carve(char *base, size_t total, int kappa, SampledScratch *out);
-// Labels every loop of the level and writes the output-side stage; raises
-// *gate if some walk exceeded `cap` hops (the level must then be relabelled).
-int sampled_label(uint4 *S, const uint32_t *Q, const SampledScratch &sc, size_t total, int log2m,
-                  int kappa, uint32_t salt, uint32_t cap, BitsLayout L, int out_stage,
+// Labels every loop of the level, writes the output-side stage and the next
+// level's records Sn; raises *gate if some walk exceeded `cap` hops (the level
+// must then be relabelled and Sn rewritten).
+int sampled_label(uint4 *S, const uint32_t *Q, uint4 *Sn, const SampledScratch &sc, size_t total,
+                  int log2m, int kappa, uint32_t salt, uint32_t cap, BitsLayout L, int out_stage,
                   uint32_t *gate, cudaStream_t s);
 // owner[0] and owner[1] must be all kUnowned before the first sampled_label.
 int sampled_scratch_reset(const SampledScratch &sc, size_t total, int kappa, cudaStream_t s);

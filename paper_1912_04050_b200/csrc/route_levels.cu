@@ -57,6 +57,68 @@ k_inverse(const uint4 *__restrict__ P4, uint4 *__restrict__ S, uint32_t *__restr
     }
 }
 
+// a1 for large inputs, as two streaming passes instead of one pass of random
+// 4-byte writes.  Q is cut into buckets of 2^kBucketLog2 consecutive entries (a
+// piece that stays in L2).  Pass 1 reads P in order, writes the switch records
+// and appends (destination, source) pairs to the bucket of the destination: a
+// CTA counts its 8192 elements per bucket in shared memory, reserves room in
+// every bucket with one global atomic per bucket, then writes its pairs there.
+// A bucket of a permutation receives exactly as many pairs as it has entries;
+// for other inputs positions wrap inside the bucket, so every access stays in
+// bounds.  Pass 2 reads the pairs bucket by bucket and scatters inside the
+// bucket's piece of Q.
+constexpr int kBucketLog2 = 18;
+constexpr int kPartChunk = 8192;
+constexpr int kPartThreads = 1024;
+
+__global__ void __launch_bounds__(kPartThreads)
+k_inverse_partition(const uint32_t *__restrict__ P, uint4 *__restrict__ S, uint2 *__restrict__ pairs,
+                    uint32_t *__restrict__ fill, uint32_t buckets, uint32_t mmask) {
+    extern __shared__ uint32_t sh[];           // count[buckets], then offset[buckets]
+    uint32_t *count = sh, *offset = sh + buckets;
+    for (uint32_t b = threadIdx.x; b < buckets; b += kPartThreads) count[b] = 0u;
+    __syncthreads();
+    const size_t j0 = size_t(blockIdx.x) * kPartChunk;
+    constexpr int kPer = kPartChunk / kPartThreads;
+    uint32_t dest[kPer], rank[kPer];
+#pragma unroll
+    for (int i = 0; i < kPer; i += 2) {
+        // two values = one switch
+        const size_t j = j0 + 2 * (size_t(i / 2) * kPartThreads + threadIdx.x);
+        const uint2 p = __ldcs(reinterpret_cast<const uint2 *>(P + j));
+        const uint32_t px = p.x & mmask, py = p.y & mmask;
+        S[j >> 1] = make_uint4(px, py, kUnowned, 0u);
+        const uint32_t base = uint32_t(j) & ~mmask;
+        dest[i] = base + px;
+        dest[i + 1] = base + py;
+        rank[i] = atomicAdd(count + (dest[i] >> kBucketLog2), 1u);
+        rank[i + 1] = atomicAdd(count + (dest[i + 1] >> kBucketLog2), 1u);
+    }
+    __syncthreads();
+    for (uint32_t b = threadIdx.x; b < buckets; b += kPartThreads)
+        offset[b] = count[b] ? atomicAdd(fill + b, count[b]) : 0u;
+    __syncthreads();
+    constexpr uint32_t kInBucket = (1u << kBucketLog2) - 1u;
+#pragma unroll
+    for (int i = 0; i < kPer; ++i) {
+        const size_t j = j0 + 2 * (size_t(i / 2) * kPartThreads + threadIdx.x) + (i & 1);
+        const uint32_t b = dest[i] >> kBucketLog2;
+        const uint32_t slot = (offset[b] + rank[i]) & kInBucket;
+        pairs[(size_t(b) << kBucketLog2) + slot] = make_uint2(dest[i], uint32_t(j) & mmask);
+    }
+}
+
+__global__ void __launch_bounds__(kThreads)
+k_inverse_scatter(const uint2 *__restrict__ pairs, uint32_t *__restrict__ Q, size_t total, uint32_t mmask) {
+    const size_t i = size_t(blockIdx.x) * kThreads + threadIdx.x;
+    if (i >= total) return;
+    const uint2 pr = __ldcs(pairs + i);
+    // the destination is forced into the bucket this pair sits in
+    constexpr uint32_t kInBucket = (1u << kBucketLog2) - 1u;
+    const size_t d = (i & ~size_t(kInBucket)) | (pr.x & kInBucket);
+    Q[d] = pr.y & mmask;
+}
+
 __device__ __forceinline__ unsigned long long jump(unsigned long long w, unsigned long long t) {
     // new nxt = t.nxt, new mn = min(w.mn, t.mn): compare the high halves.
     unsigned long long hi = (w >> 32) < (t >> 32) ? (w >> 32) : (t >> 32);
@@ -121,30 +183,35 @@ k_full_label(const uint4 *__restrict__ S, const uint32_t *__restrict__ Q,
     }
 }
 
-// in-side half of a5 + a6: input-side stage word, next level's records and Q'.
-// Position tl of the upper half-block takes P[2t or 2t+1] >> 1 of switch tl,
+// in-side half of a5 + a6: input-side stage word and Q'.  With `with_records`
+// (no sampled labelling, or its gate raised) also the next level's records:
+// position tl of the upper half-block takes P[2t or 2t+1] >> 1 of switch tl,
 // so two neighbouring threads hold the two values of one record of the next
-// level: they exchange them with a shuffle and store whole records.
+// level; they exchange them with a shuffle and store whole records.
 __global__ void __launch_bounds__(kThreads)
 k_split(const uint4 *__restrict__ S, const uint2 *__restrict__ Q2, uint4 *__restrict__ Sn,
         uint32_t *__restrict__ Qn, size_t switches, uint32_t mmask, BitsLayout L, int in_stage,
-        int out_stage) {
+        int out_stage, const uint32_t *__restrict__ gate) {
+    const bool with_records = !gate || *gate != 0u;
     size_t stride = size_t(gridDim.x) * blockDim.x;
     const uint32_t H = (mmask + 1) >> 1;
     for (size_t t = size_t(blockIdx.x) * blockDim.x + threadIdx.x; t < switches; t += stride) {
         size_t base = (2 * t) & ~size_t(mmask);
         uint32_t tl = uint32_t(t - base / 2);
-        uint4 r = __ldcs(S + t);
+        if (with_records) {
+            uint4 r = __ldcs(S + t);
+            r.x &= mmask; r.y &= mmask;
+            // colour of output 2t
+            uint32_t c = (L.bits[L.word(out_stage, t >> 5)] >> (t & 31)) & 1u;
+            uint32_t up = (c ? r.y : r.x) >> 1, lo = (c ? r.x : r.y) >> 1;
+            uint32_t got = __shfl_xor_sync(0xFFFFFFFFu, (tl & 1u) ? up : lo, 1);
+            if (tl & 1u)
+                Sn[(base >> 1) + (H >> 1) + (tl >> 1)] = make_uint4(got, lo, kUnowned, 0u);
+            else
+                Sn[(base >> 1) + (tl >> 1)] = make_uint4(up, got, kUnowned, 0u);
+        }
         uint2 q = __ldcs(Q2 + t);
-        r.x &= mmask; r.y &= mmask; q.x &= mmask; q.y &= mmask;
-        // colour of output 2t
-        uint32_t c = (L.bits[L.word(out_stage, t >> 5)] >> (t & 31)) & 1u;
-        uint32_t up = (c ? r.y : r.x) >> 1, lo = (c ? r.x : r.y) >> 1;
-        uint32_t got = __shfl_xor_sync(0xFFFFFFFFu, (tl & 1u) ? up : lo, 1);
-        if (tl & 1u)
-            Sn[(base >> 1) + (H >> 1) + (tl >> 1)] = make_uint4(got, lo, kUnowned, 0u);
-        else
-            Sn[(base >> 1) + (tl >> 1)] = make_uint4(up, got, kUnowned, 0u);
+        q.x &= mmask; q.y &= mmask;
         // colour of the output fed by input 2t
         size_t o = base + q.x;
         uint32_t cin = ((L.bits[L.word(out_stage, o >> 6)] >> ((o >> 1) & 31)) & 1u) ^ (q.x & 1u);
@@ -191,6 +258,20 @@ int cooperative_grid(int *out) {
 
 }  // namespace
 
+int launch_inverse_partitioned(const uint32_t *perm, uint4 *S, uint32_t *Q, void *pairs, uint32_t *fill,
+                               size_t total, int log2m, cudaStream_t s) {
+    const uint32_t buckets = uint32_t(total >> kBucketLog2);
+    const uint32_t mmask = (1u << log2m) - 1u;
+    BENES_CUDA_TRY(cudaMemsetAsync(fill, 0, size_t(buckets) * 4, s));
+    k_inverse_partition<<<unsigned(total / kPartChunk), kPartThreads, size_t(buckets) * 8, s>>>(
+        perm, S, static_cast<uint2 *>(pairs), fill, buckets, mmask);
+    int rc = launch_status();
+    if (rc) return rc;
+    k_inverse_scatter<<<unsigned((total + kThreads - 1) / kThreads), kThreads, 0, s>>>(
+        static_cast<const uint2 *>(pairs), Q, total, mmask);
+    return launch_status();
+}
+
 int launch_inverse(const uint32_t *perm, uint4 *S, uint32_t *Q, size_t total, int log2m,
                    cudaStream_t s) {
     size_t quads = total / 4;
@@ -220,11 +301,12 @@ int launch_full_label(const uint4 *S, const uint32_t *Q, unsigned long long *Wd,
 }
 
 int launch_split(const uint4 *S, const uint32_t *Q, uint4 *Sn, uint32_t *Qn, size_t total,
-                 int log2m, BitsLayout L, int in_stage, int out_stage, cudaStream_t s) {
+                 int log2m, BitsLayout L, int in_stage, int out_stage, const uint32_t *gate,
+                 cudaStream_t s) {
     size_t switches = total / 2;
     k_split<<<grid_for(switches), kThreads, 0, s>>>(S, reinterpret_cast<const uint2 *>(Q), Sn, Qn,
                                                     switches, (1u << log2m) - 1u, L, in_stage,
-                                                    out_stage);
+                                                    out_stage, gate);
     return launch_status();
 }
 

@@ -235,14 +235,22 @@ int launch_list_label(unsigned long long *W, uint32_t count, int beta, cudaStrea
     return launch_status();
 }
 
-// Step 5 + output side of the level's switches.
+// Step 5 + output side of the level's switches + the next level's records:
+// position tl of a half-block takes one of the two P values of switch tl, so
+// two neighbouring threads hold the two values of one record of the next
+// level; they exchange them with a shuffle and store whole records (owner
+// reset).  If the gate is raised afterwards, the split kernel redoes the
+// records from the relabelled stage.
 __global__ void __launch_bounds__(kThreads)
 k_colour(const uint4 *__restrict__ S, const uint32_t *__restrict__ Q,
-         const unsigned long long *__restrict__ W, size_t switches, uint32_t rulers, uint32_t mmask,
-         BitsLayout L, int out_stage, uint32_t cap, uint32_t *__restrict__ gate) {
+         const unsigned long long *__restrict__ W, uint4 *__restrict__ Sn, size_t switches,
+         uint32_t rulers, uint32_t mmask, BitsLayout L, int out_stage, uint32_t cap,
+         uint32_t *__restrict__ gate) {
     const size_t stride = size_t(gridDim.x) * blockDim.x;
+    const uint32_t H = (mmask + 1) >> 1;
     for (size_t t = size_t(blockIdx.x) * blockDim.x + threadIdx.x; t < switches; t += stride) {
-        const uint32_t code = __ldcs(reinterpret_cast<const uint32_t *>(S + t) + 2);
+        const uint4 r = __ldcs(S + t);
+        const uint32_t code = r.z;
         uint32_t c;
         if (code != kUnowned) {
             const uint32_t rho = code >> 1;
@@ -267,6 +275,15 @@ k_colour(const uint4 *__restrict__ S, const uint32_t *__restrict__ Q,
         }
         const uint32_t word = __ballot_sync(0xFFFFFFFFu, c);
         if ((threadIdx.x & 31) == 0) L.bits[L.word(out_stage, t >> 5)] = word;
+        const size_t base = (2 * t) & ~size_t(mmask);
+        const uint32_t tl = uint32_t(t - base / 2);
+        const uint32_t px = r.x & mmask, py = r.y & mmask;
+        const uint32_t up = (c ? py : px) >> 1, lo = (c ? px : py) >> 1;
+        const uint32_t got = __shfl_xor_sync(0xFFFFFFFFu, (tl & 1u) ? up : lo, 1);
+        if (tl & 1u)
+            Sn[(base >> 1) + (H >> 1) + (tl >> 1)] = make_uint4(got, lo, kUnowned, 0u);
+        else
+            Sn[(base >> 1) + (tl >> 1)] = make_uint4(up, got, kUnowned, 0u);
     }
 }
 
@@ -321,8 +338,8 @@ int sampled_scratch_reset(const SampledScratch &sc, size_t total, int kappa, cud
     return BENES_OK;
 }
 
-int sampled_label(uint4 *S, const uint32_t *Q, const SampledScratch &sc, size_t total, int log2m,
-                  int kappa, uint32_t salt, uint32_t cap, BitsLayout L, int out_stage,
+int sampled_label(uint4 *S, const uint32_t *Q, uint4 *Sn, const SampledScratch &sc, size_t total,
+                  int log2m, int kappa, uint32_t salt, uint32_t cap, BitsLayout L, int out_stage,
                   uint32_t *gate, cudaStream_t s) {
     const uint32_t mmask = (1u << log2m) - 1u;
     const uint32_t R = uint32_t(total >> kappa);
@@ -377,7 +394,7 @@ int sampled_label(uint4 *S, const uint32_t *Q, const SampledScratch &sc, size_t 
         size_t blocks = (switches + kThreads - 1) / kThreads;
         const size_t capb = size_t(kSMs) * 8;
         k_colour<<<unsigned(blocks < capb ? blocks : capb), kThreads, 0, s>>>(
-            S, Q, sc.list[0], switches, R, mmask, L, out_stage, cap, gate);
+            S, Q, sc.list[0], Sn, switches, R, mmask, L, out_stage, cap, gate);
         return launch_status();
     }
 }

@@ -120,6 +120,21 @@ def test_route_walks_that_give_up_fall_back_to_full_pointer_jumping(cap, labelli
         assert np.array_equal(gpu_route(perm, n), oracle.route(perm, n))
 
 
+@pytest.mark.parametrize("n,batch", [(22, 1), (16, 64), (14, 256), (15, 136), (16, 65)])
+def test_route_bucketed_inverse(n, batch):
+    """batch * N >= 2^22 in whole buckets of 2^18 takes the two-pass inverse at
+    level 0 (the last case does not and takes the plain scatter); with the option
+    off every case takes the plain scatter.  Same bits either way."""
+    perm = inputs.random_perm_batch(n, batch, seed0=3 * n) if batch > 1 else inputs.random_perm(n, 77)
+    want = oracle.route(perm, n)
+    assert np.array_equal(gpu_route(perm, n), want)
+    binding.benes_set_option(binding.OPT_INVERSE_PARTITIONED, 0)
+    try:
+        assert np.array_equal(gpu_route(perm, n), want)
+    finally:
+        binding.benes_set_option(binding.OPT_INVERSE_PARTITIONED, 1)
+
+
 # ---- apply ------------------------------------------------------------------
 @pytest.mark.parametrize("n", [1, 2, 3, 4, 5, 6, 7, 10, 12, 13, 14, 16, 19, 21])
 @pytest.mark.parametrize("dtype", [np.uint32, np.uint64])
