@@ -180,6 +180,7 @@ int launch_fused(const void *Pv, int records, size_t total, int log2m, uint32_t 
         case 11: return launch_one<11>(P, records, total, bits, log2n, s);
         case 12: return launch_one<12>(P, records, total, bits, log2n, s);
         case 13: return launch_one<13>(P, records, total, bits, log2n, s);
+        case 14: return launch_one<14>(P, records, total, bits, log2n, s);
         default: return BENES_ERR_BADARG;
     }
 }
