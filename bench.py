@@ -137,6 +137,20 @@ def gpu_index(local_rank: int) -> int:
     return local_rank
 
 
+def max_over_ranks(values, dist, device):
+    """Every rank's timings -> the slowest rank's (all ranks get the same list)."""
+    import torch
+    vals = torch.tensor(values, dtype=torch.float64, device=device)
+    if dist:
+        dist.all_reduce(vals, op=dist.ReduceOp.MAX)
+    return vals.tolist()
+
+
+def whole_job_value(elems_per_rank: int, world: int, ms_per_step: float) -> float:
+    """Elements all ranks routed per second (replicas: every rank does elems_per_rank per step)."""
+    return world * elems_per_rank / (ms_per_step * 1e-3)
+
+
 def make_inputs(name: str, rank: int):
     import numpy as np
     from paper_1912_04050_b200 import inputs
@@ -347,10 +361,7 @@ def run_gpu(args):
         assert torch.equal(out_p, d_out.cpu()), "end-to-end payload differs from the device-resident run"
 
     ms_step = ms_total / args.steps
-    vals = torch.tensor([ms_step, e2e_ms, route_ms, apply_ms], dtype=torch.float64, device="cuda")
-    if dist:
-        dist.all_reduce(vals, op=dist.ReduceOp.MAX)
-    ms_step, e2e_ms, route_ms, apply_ms = vals.tolist()
+    ms_step, e2e_ms, route_ms, apply_ms = max_over_ranks([ms_step, e2e_ms, route_ms, apply_ms], dist, "cuda")
 
     if rank == 0:
         peak, peak_kind = measured_peaks()
@@ -373,7 +384,7 @@ def run_gpu(args):
             }
         bits_bytes = d_bits.numel() * 4
         line = {
-            "metric": METRIC, "value": world * elems / (ms_step * 1e-3), "unit": UNIT,
+            "metric": METRIC, "value": whole_job_value(elems, world, ms_step), "unit": UNIT,
             "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
             "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "u32", "data": "synthetic",
