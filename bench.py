@@ -66,6 +66,7 @@ def algorithmic_bytes_per_element(kind: str, ebytes: int, kappa: int) -> float:
 # for the kernel as it stands.
 NCU_DRAM_BYTES_PER_ELEMENT = {}
 FALLBACK_HBM_GBS = 6650.0
+RANDOM_GATHER_PEAK_G = 64.7
 
 
 def measured_peaks():
@@ -382,6 +383,14 @@ def run_gpu(args):
                 "algorithmic_bytes_per_launch": bpe * elems,
                 "avg_launch_ms": per_launch_s * 1e3, "launches_timed": dom["launches"],
             }
+            if top == "walk":
+                # the walk is a chain of dependent random accesses: per switch one 16-byte
+                # record and one 4-byte inverse entry (the claim hits the record's sector)
+                acc = float(elems) / per_launch_s / 1e9
+                roofline["random_access"] = {
+                    "achieved": acc, "unit": "G accesses/s", "peak": RANDOM_GATHER_PEAK_G,
+                    "peak_source": "stand-alone test on this GPU: independent random 4-byte gathers "
+                                   "from a 256 MiB array", "frac": acc / RANDOM_GATHER_PEAK_G}
         bits_bytes = d_bits.numel() * 4
         line = {
             "metric": METRIC, "value": whole_job_value(elems, world, ms_step), "unit": UNIT,
