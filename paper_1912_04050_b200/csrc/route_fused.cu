@@ -96,15 +96,21 @@ k_route_fused(const uint32_t *__restrict__ P, int records, uint32_t *__restrict_
         }
         __syncthreads();
 
-        // a3: logS-1 passes; the last one only for even outputs
+        // a3: at most logS-1 passes; the last one only for even outputs.  A pass
+        // that changes no word has reached the fixed point (every successor's
+        // window then spans its whole cycle), and in-place updates usually get
+        // there early.
         for (int r = 1; r < logS - 1; ++r) {
+            int changed = 0;
             for (int j = tid; j < M; j += T) {
                 uint32_t w = Wd[j];
                 uint32_t v = Wd[w & 0xFFFFu];
                 uint32_t hw = w & 0xFFFF0000u, hv = v & 0xFFFF0000u;
-                Wd[j] = (hw < hv ? hw : hv) | (v & 0xFFFFu);
+                uint32_t nw = (hw < hv ? hw : hv) | (v & 0xFFFFu);
+                changed |= (nw != w);
+                Wd[j] = nw;
             }
-            __syncthreads();
+            if (!__syncthreads_or(changed)) break;
         }
         // last pass + a4 + output side of a5
         for (int t = tid; t < kPairsPadded; t += T) {

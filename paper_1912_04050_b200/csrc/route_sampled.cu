@@ -235,6 +235,17 @@ int launch_list_label(unsigned long long *W, uint32_t count, int beta, cudaStrea
     return launch_status();
 }
 
+// Between steps 4 and 5: parity of every ruler's cycle minimum, one bit each,
+// so that the colouring kernel gathers from an array 64 times smaller than
+// the list (it stays in L1/L2 next to the streaming traffic).
+__global__ void __launch_bounds__(kThreads)
+k_list_bits(const unsigned long long *__restrict__ W, uint32_t *__restrict__ cb, uint32_t rulers) {
+    const uint32_t rho = blockIdx.x * kThreads + threadIdx.x;     // rulers is a multiple of 32
+    const uint32_t bit = rho < rulers ? (uint32_t(__ldcs(W + rho) >> 32) & 1u) : 0u;
+    const uint32_t word = __ballot_sync(0xFFFFFFFFu, bit);
+    if ((threadIdx.x & 31) == 0 && rho < rulers) cb[rho >> 5] = word;
+}
+
 // Step 5 + output side of the level's switches + the next level's records:
 // position tl of a half-block takes one of the two P values of switch tl, so
 // two neighbouring threads hold the two values of one record of the next
@@ -243,7 +254,7 @@ int launch_list_label(unsigned long long *W, uint32_t count, int beta, cudaStrea
 // records from the relabelled stage.
 __global__ void __launch_bounds__(kThreads)
 k_colour(const uint4 *__restrict__ S, const uint32_t *__restrict__ Q,
-         const unsigned long long *__restrict__ W, uint4 *__restrict__ Sn, size_t switches,
+         const uint32_t *__restrict__ cb, uint4 *__restrict__ Sn, size_t switches,
          uint32_t rulers, uint32_t mmask, BitsLayout L, int out_stage, uint32_t cap,
          uint32_t *__restrict__ gate) {
     const size_t stride = size_t(gridDim.x) * blockDim.x;
@@ -254,7 +265,8 @@ k_colour(const uint4 *__restrict__ S, const uint32_t *__restrict__ Q,
         uint32_t c;
         if (code != kUnowned) {
             const uint32_t rho = code >> 1;
-            c = (uint32_t(__ldg(W + (rho < rulers ? rho : 0u)) >> 32) ^ code) & 1u;
+            const uint32_t rr = rho < rulers ? rho : 0u;
+            c = ((__ldg(cb + (rr >> 5)) >> (rr & 31u)) ^ code) & 1u;
         } else {
             // loop without ruler: walk the g-cycle of output 2t
             const uint32_t j0 = uint32_t(2 * t);
@@ -388,13 +400,18 @@ int sampled_label(uint4 *S, const uint32_t *Q, uint4 *Sn, const SampledScratch &
         int rc = launch_status();
         if (rc) return rc;
     }
+    // the walk records are dead: their memory takes the rulers' colour bits
+    uint32_t *cb = reinterpret_cast<uint32_t *>(sc.rec);
     {
         ProfileScope ps(kColour, s);
+        k_list_bits<<<rgrid, kThreads, 0, s>>>(sc.list[0], cb, R);
+        int rc = launch_status();
+        if (rc) return rc;
         const size_t switches = total / 2;
         size_t blocks = (switches + kThreads - 1) / kThreads;
         const size_t capb = size_t(kSMs) * 8;
         k_colour<<<unsigned(blocks < capb ? blocks : capb), kThreads, 0, s>>>(
-            S, Q, sc.list[0], Sn, switches, R, mmask, L, out_stage, cap, gate);
+            S, Q, cb, Sn, switches, R, mmask, L, out_stage, cap, gate);
         return launch_status();
     }
 }
