@@ -1,18 +1,31 @@
 // Fused path: one CTA finishes every remaining level of one block of size
-// M = 2^LOGM entirely in shared memory (inverse scatter, successor pairing,
-// pointer jumping, colouring, stage bits, compaction, middle stage).  It serves
-// both the tail of a large permutation (the flat level-(n-LOGM) array holds
-// N/M blocks) and a batch of small permutations (N = M, one CTA each).
+// M = 2^LOGM entirely in shared memory (inverse scatter, loop labelling,
+// colouring, stage bits, compaction, middle stage).  It serves both the tail of
+// a large permutation (the flat level-(n-LOGM) array holds N/M blocks) and a
+// batch of small permutations (N = M, one CTA each).
 //
-// Shared-memory words are 32 bit: low 16 = nxt, high 16 = mn, both indices
-// local to the CTA's block (M <= 2^16).  Passes are separated by a CTA barrier,
-// updates inside a pass are in place: a 32-bit shared-memory access is atomic,
-// and a word read at any time satisfies "mn = min over the path from j up to,
-// excluding, nxt", so every pass at least doubles the shortest window.
+// All indices are local to the CTA's block and 16 bit (M <= 2^15).  A level
+// works on sub-blocks of size S; its loops are labelled the same way as at the
+// HBM levels, with shared-memory latencies:
+//   - sub-blocks of S >= 512: one ruler switch per 8 switches; a walker per
+//     ruler output follows g, claims switches with a 16-bit compare-and-swap
+//     and stops where it meets the walker from the other end; the contracted
+//     list (M/8 words of (next, min), 16 + 16 bit) is labelled by in-place
+//     pointer jumping; a switch takes (minimum of its owner & 1) ^ side;
+//   - switches nobody claimed (loops without ruler) walk their own cycle;
+//   - sub-blocks of S <= 256 are labelled by in-place pointer jumping over all
+//     outputs with 16-bit words (next, min: 8 + 8 bit, local to the sub-block),
+//     which costs fewer instructions than walks once cycles are this short.
+// The scratch of the labelling (owners, walk records, list) lives where the
+// next level's P' is written afterwards.
 #include "common.cuh"
 
 namespace benes {
 namespace {
+
+constexpr int kFKappa = 3;                     // ruler spacing (log2) inside a CTA
+constexpr int kFMinLogS = 9;                   // smallest sub-block that is sampled; below: 8+8-bit pointer jumping
+constexpr uint32_t kNone16 = 0xFFFFu;
 
 template <int LOGM>
 struct FusedCfg {
@@ -20,9 +33,20 @@ struct FusedCfg {
     static constexpr int kPairs = M / 2;
     static constexpr int kThreads = kPairs >= 1024 ? 1024 : (kPairs >= 32 ? kPairs : 32);
     static constexpr int kColourWords = M >= 64 ? M / 64 : 1;
-    // Pa, Pb, Q: uint16[M] each; Wd: uint32[M]; colour words
-    static constexpr size_t kSmemBytes = size_t(M) * (2 + 2 + 2 + 4) + size_t(kColourWords) * 4;
+    static constexpr int kRulers = M >> kFKappa;                 // ruler outputs (0 if M < 8)
+    // Pa, Pb, Q: uint16[M]; colour words; scratch beyond Pb: see carve-up in the kernel
+    static constexpr size_t kScratchBytes = size_t(M) + size_t(kRulers) * (4 + 2 + 4);   // owners, records, list
+    static constexpr size_t kExtra = kScratchBytes > size_t(2 * M) ? kScratchBytes - size_t(2 * M) : 0;
+    static constexpr size_t kSmemBytes = size_t(M) * 6 + size_t(kColourWords) * 4 + kExtra + 16;
 };
+
+__device__ __forceinline__ uint32_t fused_slot(uint32_t group, uint32_t salt) {
+    uint32_t h = group * 0x9E3779B1u + salt;
+    h ^= h >> 15;
+    h *= 0x85EBCA6Bu;
+    h ^= h >> 13;
+    return h & ((1u << kFKappa) - 1u);
+}
 
 template <int LOGM>
 __global__ void __launch_bounds__(FusedCfg<LOGM>::kThreads)
@@ -30,15 +54,20 @@ k_route_fused(const uint32_t *__restrict__ P, int records, uint32_t *__restrict_
     using C = FusedCfg<LOGM>;
     constexpr int M = C::M;
     constexpr int T = C::kThreads;
+    constexpr int R = C::kRulers;
     // pair loops run over a multiple of 32 so that every lane reaches the ballots
     constexpr int kPairsPadded = C::kPairs >= 32 ? C::kPairs : 32;
 
     extern __shared__ __align__(16) unsigned char smem_raw[];
     uint16_t *Pa = reinterpret_cast<uint16_t *>(smem_raw);
-    uint16_t *Pb = Pa + M;
-    uint16_t *Q = Pb + M;
-    uint32_t *Wd = reinterpret_cast<uint32_t *>(Q + M);
-    uint32_t *cw = Wd + M;
+    uint16_t *Q = Pa + M;
+    uint32_t *cw = reinterpret_cast<uint32_t *>(Q + M);
+    uint16_t *Pb = reinterpret_cast<uint16_t *>(cw + C::kColourWords);   // + scratch tail
+    // Pa and Pb swap roles every level, the labelling scratch always overlays
+    // the buffer P' is written to next; it starts at that buffer's first byte.
+    // Since only Pb is followed by the extra bytes, the scratch that does not
+    // fit into 2M bytes is taken from the tail behind Pb in both cases.
+    unsigned char *tail = reinterpret_cast<unsigned char *>(Pb + M);
 
     const int tid = threadIdx.x;
     const int lane = tid & 31;
@@ -60,6 +89,7 @@ k_route_fused(const uint32_t *__restrict__ P, int records, uint32_t *__restrict_
     }
     __syncthreads();
 
+    uint16_t *Pcur = Pa, *Pnext = Pb;
 #pragma unroll 1
     for (int k = 0; k < LOGM; ++k) {
         const int logS = LOGM - k;
@@ -70,61 +100,155 @@ k_route_fused(const uint32_t *__restrict__ P, int records, uint32_t *__restrict_
         if (logS == 1) {
             // a7: middle stage, crossed iff output 0 of the 2-block takes input 1
             for (int t = tid; t < kPairsPadded; t += T) {
-                uint32_t b = (t < C::kPairs) ? (Pa[2 * t] & 1u) : 0u;
+                uint32_t b = (t < C::kPairs) ? (Pcur[2 * t] & 1u) : 0u;
                 uint32_t word = __ballot_sync(0xFFFFFFFFu, b);
                 if (lane == 0) my_bits[size_t(n - 1) * stage_w + (t >> 5)] = word;
             }
             break;
         }
 
-        // a1: block-local inverse
+        // scratch of this level's labelling: first 2M bytes = the buffer P' goes to, rest = tail
+        // owners: uint16 per switch (M bytes); records (own min | far min << 16): uint32 per ruler
+        // output; peers: uint16 per ruler output; list words (next | min << 16): uint32 per ruler
+        uint16_t *own = Pnext;
+        uint32_t *recm = reinterpret_cast<uint32_t *>(reinterpret_cast<unsigned char *>(Pnext) + M);
+        uint32_t *list = recm + R;                       // recm and list fill the second M bytes
+        uint16_t *peer = reinterpret_cast<uint16_t *>(tail);
+        const bool sampled = logS >= kFMinLogS;
+
+        // a1: block-local inverse; owners reset
         for (int j = tid; j < M; j += T) {
             uint32_t sb = uint32_t(j) & ~smask;
-            Q[sb + (Pa[j] & smask)] = uint16_t(uint32_t(j) & smask);
+            Q[sb + (Pcur[j] & smask)] = uint16_t(uint32_t(j) & smask);
         }
+        if (sampled)
+            for (int t = tid; t < C::kPairs; t += T) own[t] = uint16_t(kNone16);
         __syncthreads();
 
-        // a2: successor and initial word
-        for (int t = tid; t < C::kPairs; t += T) {
-            uint32_t j = 2u * t;
-            uint32_t sb = j & ~smask;
-            uint32_t p0 = Pa[j] & smask, p1 = Pa[j + 1] & smask;
-            uint32_t g0 = sb + (Q[sb + (p1 ^ 1u)] & smask);
-            uint32_t g1 = sb + (Q[sb + (p0 ^ 1u)] & smask);
-            Wd[j] = g0 | (j << 16);
-            Wd[j + 1] = g1 | ((j + 1u) << 16);
+        if (sampled) {
+            // walks from the ruler outputs; they meet in the middle of a segment
+            for (int rho = tid; rho < R; rho += T) {
+                const uint32_t group = uint32_t(rho) >> 1, side0 = uint32_t(rho) & 1u;
+                const uint32_t t0 = (group << kFKappa) | fused_slot(group, uint32_t(level));
+                uint32_t j = 2u * t0 + side0;
+                const uint32_t sb = j & ~smask;
+                uint32_t fwd = j, part = kNone16, pr = uint32_t(rho) ^ 1u;
+                if (!side0) own[t0] = uint16_t(rho << 1);
+                uint32_t pp = *reinterpret_cast<const uint32_t *>(Pcur + 2u * t0);
+                uint32_t p = (side0 ? pp : (pp >> 16)) & smask;            // P[j^1]
+                uint32_t q = Q[sb + (p ^ 1u)] & smask;
+                for (uint32_t hops = 0; hops < S; ++hops) {                // a walk claims < S/2 switches
+                    j = sb + q;
+                    const uint32_t t = j >> 1, side = j & 1u, g = t >> kFKappa;
+                    if ((t & ((1u << kFKappa) - 1u)) == fused_slot(g, uint32_t(level))) {
+                        pr = (2u * g + side) ^ 1u;                          // reached the next ruler
+                        break;
+                    }
+                    pp = *reinterpret_cast<const uint32_t *>(Pcur + 2u * t);
+                    p = (side ? pp : (pp >> 16)) & smask;
+                    const uint32_t qn = Q[sb + (p ^ 1u)] & smask;
+                    const uint32_t prev = atomicCAS(reinterpret_cast<unsigned short *>(own + t),
+                                                    static_cast<unsigned short>(kNone16),
+                                                    static_cast<unsigned short>((uint32_t(rho) << 1) | side));
+                    if (prev != kNone16) {                                  // met the other walker
+                        pr = prev >> 1;
+                        break;
+                    }
+                    fwd = min(fwd, j);
+                    part = min(part, j ^ 1u);
+                    q = qn;
+                }
+                recm[rho] = fwd | (part << 16);
+                peer[rho] = uint16_t(pr < uint32_t(R) ? pr : uint32_t(rho));
+            }
+            __syncthreads();
+            // contracted list: next = peer ^ 1, minimum = own side of mine, far side of the peer's
+            for (int rho = tid; rho < R; rho += T) {
+                const uint32_t pr = peer[rho];
+                const uint32_t mn = min(recm[rho] & 0xFFFFu, recm[pr] >> 16);
+                list[rho] = (pr ^ 1u) | (mn << 16);
+            }
+            __syncthreads();
+            // in-place pointer jumping over the list; a cycle of the list has at most
+            // S/16 words (half of the ruler outputs of its sub-block)
+            for (int r = 0; r < logS - kFKappa - 1; ++r) {
+                int changed = 0;
+                for (int e = tid; e < R; e += T) {
+                    uint32_t w = list[e];
+                    uint32_t v = list[w & 0xFFFFu];
+                    uint32_t hw = w & 0xFFFF0000u, hv = v & 0xFFFF0000u;
+                    uint32_t nw = (hw < hv ? hw : hv) | (v & 0xFFFFu);
+                    changed |= (nw != w);
+                    list[e] = nw;
+                }
+                if (!__syncthreads_or(changed)) break;
+            }
         }
-        __syncthreads();
 
-        // a3: at most logS-1 passes; the last one only for even outputs.  A pass
-        // that changes no word has reached the fixed point (every successor's
-        // window then spans its whole cycle), and in-place updates usually get
-        // there early.
-        for (int r = 1; r < logS - 1; ++r) {
-            int changed = 0;
-            for (int j = tid; j < M; j += T) {
-                uint32_t w = Wd[j];
-                uint32_t v = Wd[w & 0xFFFFu];
-                uint32_t hw = w & 0xFFFF0000u, hv = v & 0xFFFF0000u;
-                uint32_t nw = (hw < hv ? hw : hv) | (v & 0xFFFFu);
-                changed |= (nw != w);
-                Wd[j] = nw;
+        if (sampled) {
+            // a4 + output side of a5: colour of output 2t from its owner
+            for (int t = tid; t < kPairsPadded; t += T) {
+                uint32_t c = 0;
+                if (t < C::kPairs) {
+                    const uint32_t code = own[t];
+                    if (code != kNone16) {
+                        c = ((list[code >> 1] >> 16) ^ code) & 1u;
+                    } else {
+                        // no owner: walk the g-cycle of output 2t (at most S/2 outputs)
+                        const uint32_t j0 = 2u * uint32_t(t), sb = j0 & ~smask;
+                        uint32_t j = j0, mn = j0;
+                        for (uint32_t hops = 0; hops < S; ++hops) {
+                            const uint32_t p = Pcur[j ^ 1u] & smask;
+                            j = sb + (Q[sb + (p ^ 1u)] & smask);
+                            if (j == j0) break;
+                            mn = min(mn, j);
+                        }
+                        c = mn & 1u;
+                    }
+                }
+                uint32_t word = __ballot_sync(0xFFFFFFFFu, c);
+                if (lane == 0) {
+                    cw[t >> 5] = word;
+                    my_bits[size_t(2 * n - 2 - level) * stage_w + (t >> 5)] = word;
+                }
             }
-            if (!__syncthreads_or(changed)) break;
-        }
-        // last pass + a4 + output side of a5
-        for (int t = tid; t < kPairsPadded; t += T) {
-            uint32_t c = 0;
-            if (t < C::kPairs) {
-                uint32_t w = Wd[2 * t];
-                uint32_t v = Wd[w & 0xFFFFu];
-                uint32_t mn = (w >> 16) < (v >> 16) ? (w >> 16) : (v >> 16);
-                c = mn & 1u;
+        } else {
+            // a2: successor and initial word (next | min << 8), indices local to the sub-block
+            uint16_t *Wd = Pnext;
+            for (int t = tid; t < C::kPairs; t += T) {
+                const uint32_t j = 2u * t, sb = j & ~smask, jl = j & smask;
+                const uint32_t pp = *reinterpret_cast<const uint32_t *>(Pcur + j);
+                const uint32_t p0 = pp & smask, p1 = (pp >> 16) & smask;
+                const uint32_t g0 = Q[sb + (p1 ^ 1u)] & smask, g1 = Q[sb + (p0 ^ 1u)] & smask;
+                *reinterpret_cast<uint32_t *>(Wd + j) = (g0 | (jl << 8)) | ((g1 | ((jl + 1u) << 8)) << 16);
             }
-            uint32_t word = __ballot_sync(0xFFFFFFFFu, c);
-            if (lane == 0) {
-                cw[t >> 5] = word;
-                my_bits[size_t(2 * n - 2 - level) * stage_w + (t >> 5)] = word;
+            __syncthreads();
+            // a3: at most logS-1 passes, in place; the last one only for even outputs
+            for (int r = 1; r < logS - 1; ++r) {
+                int changed = 0;
+                for (int j = tid; j < M; j += T) {
+                    const uint32_t sb = uint32_t(j) & ~smask;
+                    const uint32_t w = Wd[j];
+                    const uint32_t v = Wd[sb + (w & 0xFFu)];
+                    const uint32_t nw = min(w & 0xFF00u, v & 0xFF00u) | (v & 0xFFu);
+                    changed |= (nw != w);
+                    Wd[j] = uint16_t(nw);
+                }
+                if (!__syncthreads_or(changed)) break;
+            }
+            for (int t = tid; t < kPairsPadded; t += T) {
+                uint32_t c = 0;
+                if (t < C::kPairs) {
+                    const uint32_t j = 2u * t, sb = j & ~smask;
+                    const uint32_t w = Wd[j];
+                    const uint32_t v = Wd[sb + (w & 0xFFu)];
+                    c = (min(w, v) >> 8) & 1u;
+                }
+                uint32_t word = __ballot_sync(0xFFFFFFFFu, c);
+                if (lane == 0) {
+                    cw[t >> 5] = word;
+                    my_bits[size_t(2 * n - 2 - level) * stage_w + (t >> 5)] = word;
+                }
             }
         }
         __syncthreads();
@@ -138,8 +262,8 @@ k_route_fused(const uint32_t *__restrict__ P, int records, uint32_t *__restrict_
                 uint32_t sb = j & ~smask;
                 uint32_t tl = (j & smask) >> 1;
                 uint32_t c = (cw[t >> 5] >> (t & 31)) & 1u;
-                Pb[sb + c * H + tl] = uint16_t((Pa[j] & smask) >> 1);
-                Pb[sb + (1u - c) * H + tl] = uint16_t((Pa[j + 1] & smask) >> 1);
+                Pnext[sb + c * H + tl] = uint16_t((Pcur[j] & smask) >> 1);
+                Pnext[sb + (1u - c) * H + tl] = uint16_t((Pcur[j + 1] & smask) >> 1);
                 uint32_t q0 = Q[j] & smask;
                 uint32_t o = sb + q0;
                 cin = ((cw[o >> 6] >> ((o >> 1) & 31)) & 1u) ^ (q0 & 1u);
@@ -148,7 +272,7 @@ k_route_fused(const uint32_t *__restrict__ P, int records, uint32_t *__restrict_
             if (lane == 0) my_bits[size_t(level) * stage_w + (t >> 5)] = word;
         }
         __syncthreads();
-        uint16_t *tmp = Pa; Pa = Pb; Pb = tmp;
+        uint16_t *tmp = Pcur; Pcur = Pnext; Pnext = tmp;
     }
 }
 
@@ -160,6 +284,9 @@ int launch_one(const uint32_t *P, int records, size_t total, uint32_t *bits, int
         BENES_CUDA_TRY(cudaFuncSetAttribute(k_route_fused<LOGM>,
                                             cudaFuncAttributeMaxDynamicSharedMemorySize,
                                             int(C::kSmemBytes)));
+        BENES_CUDA_TRY(cudaFuncSetAttribute(k_route_fused<LOGM>,
+                                            cudaFuncAttributePreferredSharedMemoryCarveout,
+                                            cudaSharedmemCarveoutMaxShared));
         configured = true;
     }
     size_t blocks = total >> LOGM;
@@ -187,6 +314,7 @@ int launch_fused(const void *Pv, int records, size_t total, int log2m, uint32_t 
         case 12: return launch_one<12>(P, records, total, bits, log2n, s);
         case 13: return launch_one<13>(P, records, total, bits, log2n, s);
         case 14: return launch_one<14>(P, records, total, bits, log2n, s);
+        case 15: return launch_one<15>(P, records, total, bits, log2n, s);
         default: return BENES_ERR_BADARG;
     }
 }
