@@ -11,7 +11,7 @@ namespace benes {
 
 // Largest block finished inside one CTA (log2).  Blocks above it go through
 // the per-level HBM kernels.
-constexpr int kFusedLog2M = 14;
+constexpr int kFusedLog2M = 15;
 
 // Largest list (log2 of its 64-bit words) that one CTA labels in shared memory.
 constexpr int kListSmemLog2 = 14;
