@@ -47,21 +47,21 @@ def gpu_apply(bits: np.ndarray, x: np.ndarray, n: int) -> np.ndarray:
 
 
 # ---- route ------------------------------------------------------------------
-@pytest.mark.parametrize("n", list(range(1, 19)))
+@pytest.mark.parametrize("n", list(range(1, 21)))
 def test_route_random_every_size(n):
-    """n = 1..13 run in one CTA; 14.. take 1.. HBM levels first, then the fused tail."""
+    """n up to benes_fused_log2m() run in one CTA; larger n take HBM levels first, then the fused tail."""
     perm = inputs.random_perm(n, 100 + n)
     assert np.array_equal(gpu_route(perm, n), oracle.route(perm, n))
 
 
-@pytest.mark.parametrize("n,batch", [(1, 5), (2, 7), (3, 33), (5, 64), (6, 3), (8, 1000), (11, 5),
-                                     (13, 3), (14, 3), (15, 2), (16, 5)])
+@pytest.mark.parametrize("n,batch", [(1, 5), (2, 7), (3, 33), (5, 64), (6, 3), (8, 1000), (9, 77), (11, 5),
+                                     (13, 3), (14, 3), (15, 2), (16, 5), (17, 3)])
 def test_route_batched(n, batch):
     perm = inputs.random_perm_batch(n, batch, seed0=7 * n)
     assert np.array_equal(gpu_route(perm, n), oracle.route(perm, n))
 
 
-@pytest.mark.parametrize("n", [4, 10, 13, 14, 16, 18])
+@pytest.mark.parametrize("n", [4, 9, 10, 13, 15, 16, 18, 20])
 @pytest.mark.parametrize("kind", ["identity", "shift1", "bitrev", "transpose", "sattolo"])
 def test_route_structured(n, kind):
     perm = inputs.structured_perms(n)[kind]
@@ -98,14 +98,14 @@ def apply_mode(request):
 def test_route_every_ruler_spacing(kappa, labelling_options):
     """0 = pointer jumping over all outputs; otherwise one ruler per 2^kappa switches."""
     binding.benes_set_option(binding.OPT_SAMPLE_LOG2K, kappa)
-    for n in (14, 17):
+    for n in (16, 19):
         perm = inputs.random_perm(n, 40 + n)
         assert np.array_equal(gpu_route(perm, n), oracle.route(perm, n))
-    n = 16
+    n = 17
     for kind, perm in inputs.structured_perms(n).items():
         assert np.array_equal(gpu_route(perm, n), oracle.route(perm, n)), kind
-    perm = inputs.random_perm_batch(15, 3, seed0=9)
-    assert np.array_equal(gpu_route(perm, 15), oracle.route(perm, 15))
+    perm = inputs.random_perm_batch(16, 3, seed0=9)
+    assert np.array_equal(gpu_route(perm, 16), oracle.route(perm, 16))
 
 
 @pytest.mark.parametrize("cap", [1, 3, 40])
@@ -113,7 +113,7 @@ def test_route_walks_that_give_up_fall_back_to_full_pointer_jumping(cap, labelli
     """With a tiny hop limit almost every level raises its gate and is relabelled
     by the full pointer-jumping kernels; the bits must not change."""
     binding.benes_set_option(binding.OPT_WALK_CAP, cap)
-    for n in (14, 16):
+    for n in (16, 18):
         for kind, perm in inputs.structured_perms(n).items():
             assert np.array_equal(gpu_route(perm, n), oracle.route(perm, n)), kind
         perm = inputs.random_perm(n, 60 + n)
@@ -231,7 +231,7 @@ def test_host_entry_points():
 
 
 def test_caller_workspace_is_used_and_checked():
-    n = 15
+    n = binding.benes_fused_log2m() + 2
     perm = inputs.random_perm(n, 11)
     need = binding.benes_route_workspace_bytes(n, 1)
     ws = torch.empty(need, dtype=torch.uint8, device="cuda")
@@ -258,7 +258,7 @@ def test_validate_perm(n, batch):
     assert not binding.benes_validate_perm(dev(bad), n, batch)
 
 
-@pytest.mark.parametrize("n", [6, 14])
+@pytest.mark.parametrize("n", [6, 14, 17, 22])
 def test_non_permutation_input_is_memory_safe(n):
     """Every index the kernels form is masked to its block, so duplicated values
     give an unspecified setting but no error; a good call afterwards is exact."""
@@ -272,7 +272,7 @@ def test_non_permutation_input_is_memory_safe(n):
 
 
 def test_launch_counter_counts():
-    n = 14
+    n = 17
     before = binding.benes_launch_count()
     gpu_route(inputs.random_perm(n, 1), n)
     after = binding.benes_launch_count()
