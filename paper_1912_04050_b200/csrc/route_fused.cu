@@ -97,6 +97,72 @@ k_route_fused(const uint32_t *__restrict__ P, int records, uint32_t *__restrict_
         const uint32_t smask = S - 1u;
         const int level = level0 + k;
 
+        if (logS == 5 && LOGM >= 5) {
+            // Sub-blocks of 32 and less stay inside one group of 32 outputs for all
+            // remaining levels: a warp finishes a group in registers, one output
+            // per lane, gathers done with shuffles (the inverse goes through 32
+            // entries of Q, which only this warp touches).
+            uint16_t *half = reinterpret_cast<uint16_t *>(my_bits);     // 16 switches = one half word
+            const size_t half_stride = stage_w * 2;
+            for (int grp = tid >> 5; grp < M / 32; grp += T / 32) {
+                const int g0 = grp * 32;
+                uint32_t p = Pcur[g0 + lane] & 31u;                      // local to the 32-sub-block
+#pragma unroll
+                for (int ls = 5; ls >= 2; --ls) {
+                    const uint32_t sm_ = (1u << ls) - 1u, sbl = uint32_t(lane) & ~sm_;
+                    const int lvl = level0 + (LOGM - ls);
+                    p &= sm_;
+                    // a1: inverse inside the sub-block
+                    Q[g0 + sbl + p] = uint16_t(uint32_t(lane) & sm_);
+                    __syncwarp();
+                    const uint32_t q = Q[g0 + lane];
+                    __syncwarp();
+                    // a2: successor
+                    const uint32_t p1 = __shfl_xor_sync(0xFFFFFFFFu, p, 1);
+                    uint32_t nxt = sbl + __shfl_sync(0xFFFFFFFFu, q, int(sbl + (p1 ^ 1u)));
+                    uint32_t mn = uint32_t(lane);
+                    // a3: synchronous pointer jumping, ls-1 passes cover cycles of 2^(ls-1)
+#pragma unroll
+                    for (int r = 0; r < ls - 1; ++r) {
+                        const uint32_t mm = __shfl_sync(0xFFFFFFFFu, mn, int(nxt));
+                        nxt = __shfl_sync(0xFFFFFFFFu, nxt, int(nxt));
+                        mn = min(mn, mm);
+                    }
+                    const uint32_t c = mn & 1u;                          // a4, every output
+                    // output side of a5: switch t = lane (< 16) takes the colour of output 2t
+                    const uint32_t ce = __shfl_sync(0xFFFFFFFFu, c, (lane & 15) * 2);
+                    const uint32_t outw = __ballot_sync(0xFFFFFFFFu, ce) & 0xFFFFu;
+                    // input side of a5: colour of the output fed by input 2t
+                    const uint32_t qe = __shfl_sync(0xFFFFFFFFu, q, (lane & 15) * 2);
+                    const uint32_t sbe = uint32_t((lane & 15) * 2) & ~sm_;
+                    const uint32_t ci = __shfl_sync(0xFFFFFFFFu, c, int(sbe + qe));
+                    const uint32_t inw = __ballot_sync(0xFFFFFFFFu, ci) & 0xFFFFu;
+                    if (lane == 0) {
+                        if (M == 32) {
+                            my_bits[size_t(2 * n - 2 - lvl) * stage_w] = outw;
+                            my_bits[size_t(lvl) * stage_w] = inw;
+                        } else {
+                            half[size_t(2 * n - 2 - lvl) * half_stride + grp] = uint16_t(outw);
+                            half[size_t(lvl) * half_stride + grp] = uint16_t(inw);
+                        }
+                    }
+                    // a6: position dl of the upper (lower) half takes the colour-0 (1) output of switch tl
+                    const uint32_t H = 1u << (ls - 1), dl = uint32_t(lane) & sm_;
+                    const uint32_t tl = dl & (H - 1u), lower = dl >> (ls - 1);
+                    const uint32_t c2 = __shfl_sync(0xFFFFFFFFu, c, int(sbl + 2u * tl));
+                    p = __shfl_sync(0xFFFFFFFFu, p, int(sbl + 2u * tl + (c2 ^ lower))) >> 1;
+                }
+                // a7: middle stage
+                const uint32_t pm = __shfl_sync(0xFFFFFFFFu, p, (lane & 15) * 2) & 1u;
+                const uint32_t midw = __ballot_sync(0xFFFFFFFFu, pm) & 0xFFFFu;
+                if (lane == 0) {
+                    if (M == 32) my_bits[size_t(n - 1) * stage_w] = midw;
+                    else half[size_t(n - 1) * half_stride + grp] = uint16_t(midw);
+                }
+            }
+            break;
+        }
+
         if (logS == 1) {
             // a7: middle stage, crossed iff output 0 of the 2-block takes input 1
             for (int t = tid; t < kPairsPadded; t += T) {
