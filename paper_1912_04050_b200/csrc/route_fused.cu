@@ -41,11 +41,8 @@ struct FusedCfg {
 };
 
 __device__ __forceinline__ uint32_t fused_slot(uint32_t group, uint32_t salt) {
-    uint32_t h = group * 0x9E3779B1u + salt;
-    h ^= h >> 15;
-    h *= 0x85EBCA6Bu;
-    h ^= h >> 13;
-    return h & ((1u << kFKappa) - 1u);
+    // top bits of a multiplicative hash: two instructions on the walk's critical path
+    return ((group + salt * 0x632BE5ABu) * 0x9E3779B1u) >> (32 - kFKappa);
 }
 
 template <int LOGM>
