@@ -35,7 +35,12 @@ WORKLOADS = {
     "c2": (8, 16384, 4, 0, "C2: 16384 x N=2^8 uniform random permutations (seeds 0..16383), route + uint32 payload apply"),
     "r25": (25, 1, 8, 2, "profiling case: 1 x N=2^25 uniform random permutation (seed 2), route + uint64 payload apply"),
     "c5s": (24, 1, 4, 3, "C5: 1 x N=2^24 Sattolo single-cycle permutation (seed 3), route + uint32 payload apply"),
+    "c5i": (24, 1, 4, 0, "C5: 1 x N=2^24 identity, route + uint32 payload apply"),
+    "c5h": (24, 1, 4, 0, "C5: 1 x N=2^24 cyclic shift by 1, route + uint32 payload apply"),
+    "c5b": (24, 1, 4, 0, "C5: 1 x N=2^24 bit reversal, route + uint32 payload apply"),
+    "c5t": (24, 1, 4, 0, "C5: 1 x N=2^24 index map of a 4096x4096 transpose, route + uint32 payload apply"),
 }
+STRUCTURED = {"c5i": "identity", "c5h": "shift1", "c5b": "bitrev", "c5t": "transpose"}
 
 def algorithmic_bytes_per_element(kind: str, ebytes: int, kappa: int) -> float:
     """Useful bytes one launch of a kernel kind moves per permutation element."""
@@ -162,6 +167,8 @@ def make_inputs(name: str, rank: int):
     n, batch, ebytes, seed, _ = WORKLOADS[name]
     if name == "c5s":
         perm = inputs.sattolo_perm(n, seed + rank)
+    elif name in STRUCTURED:
+        perm = inputs.structured_perms(n)[STRUCTURED[name]]
     elif batch == 1:
         perm = inputs.random_perm(n, seed + rank)
     else:
