@@ -1,9 +1,8 @@
 /*
  * benes.h -- C ABI of the B200 (sm_100a) Benes-network routing library.
  *
- * Problem statement (the build contract; the mounted paper has no passage on
- * it): a rearrangeable Benes network of N = 2^n inputs has 2n-1 stages of N/2
- * two-by-two switches.  benes_route computes the switch settings that make it
+ * Problem statement: a rearrangeable Benes network of N = 2^n inputs has 2n-1
+ * stages of N/2 two-by-two switches.  benes_route computes the switch settings that make it
  * realise a permutation pi given in GATHER form, out[j] = in[pi[j]];
  * benes_apply pushes a payload through the stages.
  *

@@ -6,12 +6,12 @@
  * CUDA path and must never be linked or imported by it.  Only tests, the smoke
  * check and the benchmark's CPU-baseline leg may call it.
  *
- * What it follows: the problem statement of the build contract (a
+ * What it follows: the problem statement (a
  * rearrangeable Benes network of N = 2^n inputs must realise a permutation pi
  * in gather form, out[j] = in[pi[j]]) and the classical sequential "looping
  * algorithm": walk every constraint loop once, colour its elements
  * alternately, set the outermost two stages, recurse on the two half-size
- * sub-permutations.  The mounted paper contains no statement of this method,
+ * sub-permutations.  The paper contains no statement of this method,
  * so every convention is written out here:
  *
  *   - A level l (0 <= l <= n-1) consists of 2^l independent sub-networks
