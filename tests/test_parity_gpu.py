@@ -217,6 +217,32 @@ def test_config4_n2p26_u64_payload():
     assert np.array_equal(bits, oracle.route(perm, n))
 
 
+def test_route_n2p28_properties():
+    """Beyond what the oracle finishes in reasonable time: the routed identity
+    payload must reproduce the permutation, and under the canonical rule the
+    first output switch of every block of every level is straight (output 0 of a
+    block is the smallest output of its loop)."""
+    n = 28
+    perm = inputs.random_perm(n, 5)
+    d_perm = dev(perm)
+    bits = torch.empty(binding.benes_switch_words(n, 1), dtype=torch.int32, device="cuda")
+    binding.benes_route(d_perm, n, 1, bits)
+    ident = torch.arange(1 << n, dtype=torch.int32, device="cuda")
+    out = torch.empty_like(ident)
+    binding.benes_apply_ex(bits, ident, out, 4, n, 1)
+    torch.cuda.synchronize()
+    assert torch.equal(out, d_perm)
+    del ident, out, d_perm
+    W = (1 << n) // 64
+    b = host(bits, np.uint32).reshape(2 * n - 1, W)
+    for level in range(n - 1):
+        half = (1 << (n - level)) // 2                  # switches per block
+        first = np.arange(1 << level, dtype=np.int64) * half
+        stage = b[2 * n - 2 - level]
+        assert not ((stage[first >> 5] >> (first & 31).astype(np.uint32)) & 1).any(), level
+    binding.benes_release_workspace()
+
+
 # ---- host-buffer entry points, validation, robustness -------------------------------------------
 def test_host_entry_points():
     n, batch = 15, 2
