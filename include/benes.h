@@ -149,7 +149,9 @@ int benes_validate_perm(const uint32_t *perm, int log2n, int batch, benes_stream
  *   BENES_OPT_SAMPLE_LOG2K : 0 = label every loop by pointer jumping over all
  *       outputs; kappa in 2..8 (default 4) = label only one sampled "ruler"
  *       switch per 2^kappa switches by pointer jumping and reach the rest by
- *       sequential walks between rulers.  The result is identical either way.
+ *       sequential walks between rulers (for batch * N <= 2^22 at most 2^3: short
+ *       walks matter more than short lists there).  The result is identical
+ *       either way.
  *   BENES_OPT_WALK_CAP : hops (1 .. 2^24, default 2^14) after which a walk gives
  *       up; a level in which that happens is relabelled by full pointer jumping.
  *   BENES_OPT_APPLY_FUSED : 1 (default) = benes_apply / benes_apply_ex run up to

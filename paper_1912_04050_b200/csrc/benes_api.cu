@@ -106,7 +106,9 @@ int route_levels(const uint32_t *perm, int n, size_t batch, uint32_t *bits, char
     char *sampled = ws + off; off += align_up(sampled_scratch_bytes(T, kMinKappa));
     uint32_t *gates = reinterpret_cast<uint32_t *>(ws + off); off += align_up(kMaxLevels * 4);
     uint32_t *fill = reinterpret_cast<uint32_t *>(ws + off);
-    const int kappa = g_kappa;
+    // Small inputs are bound by the longest walk of a level, not by throughput:
+    // closer rulers (shorter walks) pay there although the lists get longer.
+    const int kappa = (g_kappa > 3 && T <= (size_t(1) << 22)) ? 3 : g_kappa;
     const uint32_t cap = uint32_t(g_walk_cap);
     SampledScratch sc;
     int rc;
