@@ -394,11 +394,14 @@ def run_gpu(args):
                 "algorithmic_bytes_per_launch": bpe * elems,
                 "avg_launch_ms": per_launch_s * 1e3, "launches_timed": dom["launches"],
             }
-            if top == "walk":
+            if top == "walk" and per_level.get("walk"):
                 # the walk is a chain of dependent random accesses: per switch one 16-byte
-                # record and one 4-byte inverse entry (the claim hits the record's sector)
-                acc = float(elems) / per_launch_s / 1e9
+                # record and one 4-byte inverse entry (the claim hits the record's sector),
+                # i.e. one access per element.  Level 0 is the launch whose block (12 B per
+                # output) is furthest above the L2, so its accesses all go to DRAM.
+                acc = float(elems) / (per_level["walk"][0] * 1e-3) / 1e9
                 roofline["random_access"] = {
+                    "launch": "level 0", "ms": per_level["walk"][0],
                     "achieved": acc, "unit": "G accesses/s", "peak": RANDOM_GATHER_PEAK_G,
                     "peak_source": "stand-alone test on this GPU: independent random 4-byte gathers "
                                    "from a 256 MiB array", "frac": acc / RANDOM_GATHER_PEAK_G}
