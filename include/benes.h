@@ -160,6 +160,9 @@ int benes_validate_perm(const uint32_t *perm, int log2n, int batch, benes_stream
  *   BENES_OPT_INVERSE_PARTITIONED : 1 (default) = for batch * N >= 2^22 the inverse
  *       permutation of level 0 is formed by bucketing (destination, source)
  *       pairs and scattering bucket by bucket; 0 = one pass of random writes.
+ *   BENES_OPT_CHUNK_LOG2 : 16..30 (default 30): a batch whose levels do not fit one
+ *       CTA is processed in chunks of at most 2^value elements (whole
+ *       permutations, at least one); bounds the workspace of a large batch.
  * benes_set_option returns BENES_OK or BENES_ERR_BADARG; benes_get_option
  * returns the value, or BENES_ERR_BADARG for an unknown key.
  */
@@ -167,6 +170,7 @@ int benes_validate_perm(const uint32_t *perm, int log2n, int batch, benes_stream
 #define BENES_OPT_WALK_CAP 1
 #define BENES_OPT_APPLY_FUSED 2
 #define BENES_OPT_INVERSE_PARTITIONED 3
+#define BENES_OPT_CHUNK_LOG2 4
 int benes_set_option(int key, int value);
 int benes_get_option(int key);
 

@@ -189,6 +189,7 @@ OPT_SAMPLE_LOG2K = 0
 OPT_WALK_CAP = 1
 OPT_APPLY_FUSED = 2
 OPT_INVERSE_PARTITIONED = 3
+OPT_CHUNK_LOG2 = 4
 
 
 def benes_set_option(key: int, value: int) -> None:

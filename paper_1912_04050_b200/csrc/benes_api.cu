@@ -10,7 +10,7 @@ namespace {
 constexpr int kMaxDevices = 64;
 constexpr size_t kAlign = 256;
 // Flat elements processed together by the per-level path (indices are 32 bit).
-constexpr size_t kMaxFlat = size_t(1) << 30;
+int g_chunk_log2 = 30;
 
 struct Workspace {
     void *own = nullptr;       // library-owned buffer
@@ -70,7 +70,7 @@ inline size_t stage_words(int log2n) { return log2n >= 6 ? (size_t(1) << (log2n 
 
 // permutations per chunk of the per-level path
 inline size_t level_chunk(int log2n, size_t batch) {
-    size_t per = kMaxFlat >> log2n;
+    size_t per = (size_t(1) << g_chunk_log2) >> log2n;
     if (per < 1) per = 1;
     return batch < per ? batch : per;
 }
@@ -359,6 +359,10 @@ int benes_set_option(int key, int value) {
             if (value != 0 && value != 1) return BENES_ERR_BADARG;
             g_inverse_partitioned = value;
             return BENES_OK;
+        case BENES_OPT_CHUNK_LOG2:
+            if (value < 16 || value > 30) return BENES_ERR_BADARG;
+            g_chunk_log2 = value;
+            return BENES_OK;
         default: return BENES_ERR_BADARG;
     }
 }
@@ -370,6 +374,7 @@ int benes_get_option(int key) {
         case BENES_OPT_WALK_CAP: return g_walk_cap;
         case BENES_OPT_APPLY_FUSED: return g_apply_fused;
         case BENES_OPT_INVERSE_PARTITIONED: return g_inverse_partitioned;
+        case BENES_OPT_CHUNK_LOG2: return g_chunk_log2;
         default: return BENES_ERR_BADARG;
     }
 }

@@ -217,6 +217,24 @@ def test_config4_n2p26_u64_payload():
     assert np.array_equal(bits, oracle.route(perm, n))
 
 
+def test_route_batch_in_chunks():
+    """A batch larger than the chunk limit is routed chunk by chunk (whole
+    permutations per chunk) with a workspace sized for one chunk."""
+    n, batch = 16, 7
+    perm = inputs.random_perm_batch(n, batch, seed0=21)
+    want = oracle.route(perm, n)
+    full = binding.benes_route_workspace_bytes(n, batch)
+    binding.benes_set_option(binding.OPT_CHUNK_LOG2, 17)            # two permutations per chunk
+    try:
+        assert binding.benes_route_workspace_bytes(n, batch) < full / 3
+        assert np.array_equal(gpu_route(perm, n), want)
+        binding.benes_set_option(binding.OPT_CHUNK_LOG2, 16)        # one per chunk
+        assert np.array_equal(gpu_route(perm, n), want)
+    finally:
+        binding.benes_set_option(binding.OPT_CHUNK_LOG2, 30)
+    assert np.array_equal(gpu_route(perm, n), want)
+
+
 def test_route_n2p28_properties():
     """Beyond what the oracle finishes in reasonable time: the routed identity
     payload must reproduce the permutation, and under the canonical rule the
