@@ -176,7 +176,9 @@ k_route_fused(const uint32_t *__restrict__ P, int records, uint32_t *__restrict_
         uint16_t *own = Pnext;
         uint32_t *recm = reinterpret_cast<uint32_t *>(reinterpret_cast<unsigned char *>(Pnext) + M);
         uint32_t *list = recm + R;                       // recm and list fill the second M bytes
-        uint16_t *peer = reinterpret_cast<uint16_t *>(tail);
+        uint16_t *peer = (size_t(M) + size_t(R) * 10 <= size_t(2 * M))
+                             ? reinterpret_cast<uint16_t *>(list + R)      // still inside that buffer
+                             : reinterpret_cast<uint16_t *>(tail);
         const bool sampled = logS >= kFMinLogS;
 
         // a1: block-local inverse; owners reset
