@@ -84,6 +84,23 @@ int benes_apply_ex(const uint32_t *switch_bits, const void *in, void *out, int e
                    int log2n, int batch, benes_stream_t stream);
 
 /*
+ * Sizes that are not a power of two.  A permutation of [0, n_elems) is routed
+ * through the network of N = 2^log2n inputs, log2n = benes_padded_log2n(n_elems)
+ * (the smallest with N >= n_elems; 0 if n_elems is 0 or above 2^30), extended
+ * by fixed points pi[j] = j for j >= n_elems.
+ *   perm        : batch x n_elems uint32, each row a permutation of [0, n_elems).
+ *   switch_bits : sized and laid out for (log2n, batch), see benes_switch_words.
+ *   in, out     : batch x n_elems elements of elem_bytes (4 or 8); no overlap.
+ * out[b][j] = in[b][pi_b[j]] for j < n_elems.  Padded copies live in the
+ * library workspace.
+ */
+int benes_padded_log2n(size_t n_elems);
+int benes_route_padded(const uint32_t *perm, size_t n_elems, int batch, uint32_t *switch_bits,
+                       benes_stream_t stream);
+int benes_apply_padded(const uint32_t *switch_bits, const void *in, void *out, int elem_bytes,
+                       size_t n_elems, int batch, benes_stream_t stream);
+
+/*
  * benes_apply_ex for callers that cannot allocate device memory.  (The paper
  * has no counterpart; this is a deployment convenience of this library.)
  *

@@ -31,6 +31,9 @@ SYMBOLS = {
     "benes_apply": (_i, [_vp, _vp, _vp, _i, _i, _vp]),
     "benes_apply_ex": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp]),
     "benes_apply_static": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp]),
+    "benes_padded_log2n": (_i, [_sz]),
+    "benes_route_padded": (_i, [_vp, _sz, _i, _vp, _vp]),
+    "benes_apply_padded": (_i, [_vp, _vp, _vp, _i, _sz, _i, _vp]),
     "benes_route_host": (_i, [_vp, _i, _i, _vp, _vp]),
     "benes_apply_host": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp]),
     "benes_switch_words": (_sz, [_i, _i]),
@@ -143,6 +146,23 @@ def benes_apply_static(switch_bits: torch.Tensor, inp: torch.Tensor, out: torch.
     _check(load().benes_apply_static(_dev_ptr(switch_bits, "switch_bits"), _dev_ptr(inp, "in"),
                                      _dev_ptr(out, "out"), elem_bytes, log2n, batch, _stream(stream)),
            "benes_apply_static")
+
+
+def benes_padded_log2n(n_elems: int) -> int:
+    return load().benes_padded_log2n(n_elems)
+
+
+def benes_route_padded(perm: torch.Tensor, n_elems: int, batch: int, switch_bits: torch.Tensor, stream=None) -> None:
+    _check(load().benes_route_padded(_dev_ptr(perm, "perm"), n_elems, batch,
+                                     _dev_ptr(switch_bits, "switch_bits"), _stream(stream)),
+           "benes_route_padded")
+
+
+def benes_apply_padded(switch_bits: torch.Tensor, inp: torch.Tensor, out: torch.Tensor, elem_bytes: int,
+                       n_elems: int, batch: int, stream=None) -> None:
+    _check(load().benes_apply_padded(_dev_ptr(switch_bits, "switch_bits"), _dev_ptr(inp, "in"),
+                                     _dev_ptr(out, "out"), elem_bytes, n_elems, batch, _stream(stream)),
+           "benes_apply_padded")
 
 
 def benes_route_host(perm_host, log2n: int, batch: int, switch_bits_host, stream=None) -> None:

@@ -275,6 +275,46 @@ int benes_apply(const uint32_t *switch_bits, const void *in, void *out, int log2
     return benes_apply_ex(switch_bits, in, out, 4, log2n, batch, stream);
 }
 
+int benes_padded_log2n(size_t n_elems) {
+    if (n_elems < 1 || n_elems > (size_t(1) << BENES_MAX_LOG2N)) return 0;
+    int n = 1;
+    while ((size_t(1) << n) < n_elems) ++n;
+    return n;
+}
+
+int benes_route_padded(const uint32_t *perm, size_t n_elems, int batch, uint32_t *switch_bits,
+                       benes_stream_t stream) {
+    const int n = benes_padded_log2n(n_elems);
+    if (!perm || !switch_bits || n == 0 || batch < 1) return BENES_ERR_BADARG;
+    if ((size_t(1) << n) == n_elems) return benes_route(perm, n, batch, switch_bits, stream);
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    const size_t inner = align_up(route_ws_bytes(n, size_t(batch)));
+    void *ws = nullptr;
+    int rc = get_workspace(inner + align_up((size_t(batch) << n) * 4), &ws);
+    if (rc) return rc;
+    uint32_t *padded = reinterpret_cast<uint32_t *>(static_cast<char *>(ws) + inner);
+    if ((rc = launch_pad_perm(perm, padded, n_elems, n, size_t(batch), s))) return rc;
+    return benes_route(padded, n, batch, switch_bits, stream);
+}
+
+int benes_apply_padded(const uint32_t *switch_bits, const void *in, void *out, int elem_bytes,
+                       size_t n_elems, int batch, benes_stream_t stream) {
+    const int n = benes_padded_log2n(n_elems);
+    if (!switch_bits || !in || !out || in == out || n == 0 || batch < 1) return BENES_ERR_BADARG;
+    if (elem_bytes != 4 && elem_bytes != 8) return BENES_ERR_BADARG;
+    if ((size_t(1) << n) == n_elems) return benes_apply_ex(switch_bits, in, out, elem_bytes, n, batch, stream);
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    const size_t inner = align_up(apply_ws_bytes(elem_bytes, n, size_t(batch)));
+    const size_t row_bytes = align_up((size_t(batch) << n) * size_t(elem_bytes));
+    void *ws = nullptr;
+    int rc = get_workspace(inner + 2 * row_bytes, &ws);
+    if (rc) return rc;
+    char *pin = static_cast<char *>(ws) + inner, *pout = pin + row_bytes;
+    if ((rc = launch_pad_rows(in, pin, elem_bytes, true, n_elems, n, size_t(batch), s))) return rc;
+    if ((rc = benes_apply_ex(switch_bits, pin, pout, elem_bytes, n, batch, stream))) return rc;
+    return launch_pad_rows(pout, out, elem_bytes, false, n_elems, n, size_t(batch), s);
+}
+
 int benes_route_host(const uint32_t *perm_host, int log2n, int batch, uint32_t *switch_bits_host,
                      benes_stream_t stream) {
     if (!perm_host || !switch_bits_host || bad_shape(log2n, batch)) return BENES_ERR_BADARG;

@@ -136,6 +136,12 @@ int apply_fused_passes(int log2n);
 int launch_apply_fused(const uint32_t *bits, const void *in, void *out, void *scratch, int elem_bytes,
                        int log2n, size_t batch, cudaStream_t s);
 
+// ---- sizes that are not a power of two (pad.cu) ------------------------------
+int launch_pad_perm(const uint32_t *src, uint32_t *dst, size_t n_elems, int log2n, size_t batch,
+                    cudaStream_t s);
+int launch_pad_rows(const void *src, void *dst, int elem_bytes, bool pad, size_t n_elems, int log2n,
+                    size_t batch, cudaStream_t s);
+
 // ---- validation (route_levels.cu) -------------------------------------------
 int launch_validate(const uint32_t *perm, size_t total, int log2n, uint32_t *seen_words,
                     uint32_t *flag, cudaStream_t s);

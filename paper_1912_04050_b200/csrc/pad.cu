@@ -1,0 +1,75 @@
+// Sizes that are not a power of two: a permutation of [0, n_elems) is extended
+// to N = 2^log2n by fixed points (pi[j] = j for j >= n_elems), which leaves
+// the routing of the first n_elems positions unchanged; payloads are copied
+// into and out of rows of N elements.
+#include "common.cuh"
+
+namespace benes {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kSMs = 148;
+
+inline unsigned grid_for(size_t items) {
+    size_t blocks = (items + kThreads - 1) / kThreads;
+    size_t cap = size_t(kSMs) * 16;
+    return unsigned(blocks < cap ? (blocks ? blocks : 1) : cap);
+}
+
+// dst[b][j] = src[b][j] for j < n_elems, j for n_elems <= j < N
+__global__ void __launch_bounds__(kThreads)
+k_pad_perm(const uint32_t *__restrict__ src, uint32_t *__restrict__ dst, size_t n_elems, int log2n,
+           size_t total) {
+    const size_t stride = size_t(gridDim.x) * blockDim.x;
+    const size_t nmask = (size_t(1) << log2n) - 1;
+    for (size_t i = size_t(blockIdx.x) * blockDim.x + threadIdx.x; i < total; i += stride) {
+        const size_t b = i >> log2n, j = i & nmask;
+        dst[i] = j < n_elems ? src[b * n_elems + j] : uint32_t(j);
+    }
+}
+
+// rows of n_elems elements <-> rows of N elements (the tail of a padded row is zero)
+template <typename E, bool PAD>
+__global__ void __launch_bounds__(kThreads)
+k_pad_rows(const E *__restrict__ src, E *__restrict__ dst, size_t n_elems, int log2n, size_t total) {
+    const size_t stride = size_t(gridDim.x) * blockDim.x;
+    const size_t nmask = (size_t(1) << log2n) - 1;
+    for (size_t i = size_t(blockIdx.x) * blockDim.x + threadIdx.x; i < total; i += stride) {
+        const size_t b = i >> log2n, j = i & nmask;
+        if (PAD) dst[i] = j < n_elems ? src[b * n_elems + j] : E(0);
+        else if (j < n_elems) dst[b * n_elems + j] = src[i];
+    }
+}
+
+}  // namespace
+
+int launch_pad_perm(const uint32_t *src, uint32_t *dst, size_t n_elems, int log2n, size_t batch,
+                    cudaStream_t s) {
+    const size_t total = batch << log2n;
+    k_pad_perm<<<grid_for(total), kThreads, 0, s>>>(src, dst, n_elems, log2n, total);
+    return launch_status();
+}
+
+int launch_pad_rows(const void *src, void *dst, int elem_bytes, bool pad, size_t n_elems, int log2n,
+                    size_t batch, cudaStream_t s) {
+    const size_t total = batch << log2n;
+    const unsigned grid = grid_for(total);
+    if (elem_bytes == 4) {
+        if (pad) k_pad_rows<uint32_t, true><<<grid, kThreads, 0, s>>>(
+            static_cast<const uint32_t *>(src), static_cast<uint32_t *>(dst), n_elems, log2n, total);
+        else k_pad_rows<uint32_t, false><<<grid, kThreads, 0, s>>>(
+            static_cast<const uint32_t *>(src), static_cast<uint32_t *>(dst), n_elems, log2n, total);
+    } else if (elem_bytes == 8) {
+        if (pad) k_pad_rows<unsigned long long, true><<<grid, kThreads, 0, s>>>(
+            static_cast<const unsigned long long *>(src), static_cast<unsigned long long *>(dst), n_elems,
+            log2n, total);
+        else k_pad_rows<unsigned long long, false><<<grid, kThreads, 0, s>>>(
+            static_cast<const unsigned long long *>(src), static_cast<unsigned long long *>(dst), n_elems,
+            log2n, total);
+    } else {
+        return BENES_ERR_BADARG;
+    }
+    return launch_status();
+}
+
+}  // namespace benes

@@ -55,6 +55,24 @@ def random_perm(log2n: int, seed: int) -> np.ndarray:
     return p
 
 
+def random_perm_any(n_elems: int, batch: int, seed0: int = 0) -> np.ndarray:
+    """(batch, n_elems) uniform permutations of [0, n_elems) for any n_elems >= 1
+    (the same Fisher-Yates generator; seeds seed0 .. seed0+batch-1)."""
+    p = np.empty((batch, n_elems), dtype=np.uint32)
+    for b in range(batch):
+        _load().gen_fisher_yates(p[b].ctypes.data, n_elems, seed0 + b)
+    return p
+
+
+def pad_with_fixed_points(perm: np.ndarray, log2n: int) -> np.ndarray:
+    """Rows of n_elems values -> rows of 2^log2n values, pi[j] = j beyond n_elems."""
+    perm = np.atleast_2d(perm)
+    N = 1 << log2n
+    out = np.tile(np.arange(N, dtype=np.uint32), (perm.shape[0], 1))
+    out[:, :perm.shape[1]] = perm
+    return out
+
+
 def random_perm_batch(log2n: int, batch: int, seed0: int = 0) -> np.ndarray:
     """(batch, N) independent uniform permutations, seeds seed0 .. seed0+batch-1."""
     N = 1 << log2n

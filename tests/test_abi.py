@@ -82,6 +82,14 @@ def test_options_are_validated(lib):
     assert lib.benes_get_option(binding.OPT_SAMPLE_LOG2K) == k0 and lib.benes_get_option(binding.OPT_WALK_CAP) == c0
 
 
+def test_padded_size(lib):
+    assert [lib.benes_padded_log2n(v) for v in (1, 2, 3, 4, 5, 1024, 1025, 1 << 30)] == [1, 1, 2, 2, 3, 10, 11, 30]
+    assert lib.benes_padded_log2n(0) == 0 and lib.benes_padded_log2n((1 << 30) + 1) == 0
+    one = ctypes.c_void_p(256)
+    assert lib.benes_route_padded(one, 0, 1, one, None) == binding.BENES_ERR_BADARG
+    assert lib.benes_apply_padded(one, one, ctypes.c_void_p(512), 3, 100, 1, None) == binding.BENES_ERR_BADARG
+
+
 def test_status_strings(lib):
     assert binding.status_string(0) == "ok"
     seen = {binding.status_string(s) for s in (0, -1, -2, -3, -4)}

@@ -217,6 +217,27 @@ def test_config4_n2p26_u64_payload():
     assert np.array_equal(bits, oracle.route(perm, n))
 
 
+@pytest.mark.parametrize("n_elems,batch", [(1, 2), (3, 4), (5, 3), (100, 5), (1000, 2), (4097, 3),
+                                           (40000, 2), (100000, 1), (300001, 1)])
+def test_sizes_that_are_not_a_power_of_two(n_elems, batch):
+    """The padded entry points equal routing the permutation extended by fixed
+    points, and the routed payload is the gather of the first n_elems elements."""
+    n = binding.benes_padded_log2n(n_elems)
+    assert (1 << n) >= n_elems and (n == 1 or (1 << (n - 1)) < n_elems)
+    perm = inputs.random_perm_any(n_elems, batch, seed0=n_elems)
+    want = oracle.route(inputs.pad_with_fixed_points(perm, n), n)
+    bits = torch.full((binding.benes_switch_words(n, batch),), -1, dtype=torch.int32, device="cuda")
+    binding.benes_route_padded(dev(perm), n_elems, batch, bits)
+    torch.cuda.synchronize()
+    assert np.array_equal(host(bits, np.uint32).reshape(want.shape), want)
+    for dtype in (np.uint32, np.uint64):
+        x = np.random.default_rng(n_elems).integers(0, 2 ** 63, size=(batch, n_elems), dtype=np.uint64).astype(dtype)
+        out = torch.empty_like(dev(x))
+        binding.benes_apply_padded(bits, dev(x), out, x.dtype.itemsize, n_elems, batch)
+        torch.cuda.synchronize()
+        assert np.array_equal(host(out, dtype).reshape(x.shape), np.take_along_axis(x, perm.astype(np.int64), axis=1))
+
+
 def test_route_batch_in_chunks():
     """A batch larger than the chunk limit is routed chunk by chunk (whole
     permutations per chunk) with a workspace sized for one chunk."""
