@@ -35,6 +35,9 @@ WORKLOADS = {
     "c2": (8, 16384, 4, 0, "C2: 16384 x N=2^8 uniform random permutations (seeds 0..16383), route + uint32 payload apply"),
     "r25": (25, 1, 8, 2, "profiling case: 1 x N=2^25 uniform random permutation (seed 2), route + uint64 payload apply"),
     "c5s": (24, 1, 4, 3, "C5: 1 x N=2^24 Sattolo single-cycle permutation (seed 3), route + uint32 payload apply"),
+    "m10": (10, 16384, 4, 0, "mid-size batch: 16384 x N=2^10 uniform random permutations, route + uint32 payload apply"),
+    "m12": (12, 4096, 4, 0, "mid-size batch: 4096 x N=2^12 uniform random permutations, route + uint32 payload apply"),
+    "m16": (16, 256, 4, 0, "mid-size batch: 256 x N=2^16 uniform random permutations, route + uint32 payload apply"),
     "c5i": (24, 1, 4, 0, "C5: 1 x N=2^24 identity, route + uint32 payload apply"),
     "c5h": (24, 1, 4, 0, "C5: 1 x N=2^24 cyclic shift by 1, route + uint32 payload apply"),
     "c5b": (24, 1, 4, 0, "C5: 1 x N=2^24 bit reversal, route + uint32 payload apply"),
