@@ -238,6 +238,18 @@ def test_sizes_that_are_not_a_power_of_two(n_elems, batch):
         assert np.array_equal(host(out, dtype).reshape(x.shape), np.take_along_axis(x, perm.astype(np.int64), axis=1))
 
 
+@pytest.mark.parametrize("n", [17, 19, 21])
+def test_route_many_seeds_and_repeats(n):
+    """The walks claim switches with atomics in whatever order the hardware runs
+    them; the result must not depend on that order: several seeds, each routed
+    three times."""
+    for seed in range(6):
+        perm = inputs.random_perm(n, 1000 * n + seed)
+        want = oracle.route(perm, n)
+        for _ in range(3):
+            assert np.array_equal(gpu_route(perm, n), want), (n, seed)
+
+
 def test_route_batch_in_chunks():
     """A batch larger than the chunk limit is routed chunk by chunk (whole
     permutations per chunk) with a workspace sized for one chunk."""
