@@ -101,6 +101,18 @@ int benes_apply_padded(const uint32_t *switch_bits, const void *in, void *out, i
                        size_t n_elems, int batch, benes_stream_t stream);
 
 /*
+ * The same settings for the network drawn in place (no wiring between stages):
+ * row r of butterfly_bits pairs positions u and u | 2^i that differ in bit i,
+ * i = r for r <= n-1 and i = 2n-2-r after the middle; pair p of a row (u with
+ * bit i taken out) is bit (p & 31) of word (p >> 5); a set bit swaps the two
+ * positions.  Running the 2n-1 rows in order on a payload in place leaves
+ * out[j] = in[pi[j]].  Same size as switch_bits (benes_switch_words); the two
+ * buffers must be different.
+ */
+int benes_export_butterfly(const uint32_t *switch_bits, uint32_t *butterfly_bits, int log2n, int batch,
+                           benes_stream_t stream);
+
+/*
  * benes_apply_ex for callers that cannot allocate device memory.  (The paper
  * has no counterpart; this is a deployment convenience of this library.)
  *

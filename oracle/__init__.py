@@ -100,3 +100,54 @@ def apply(bits: np.ndarray, x: np.ndarray, log2n: int) -> np.ndarray:
     if rc != 0:
         raise RuntimeError("oracle_apply_batch failed (%d)" % rc)
     return out.reshape(x.shape)
+
+
+def _stage_bits(bits_row: np.ndarray, count: int) -> np.ndarray:
+    """First `count` bits of one stage row (LSB-first 32-bit words) as a 0/1 array."""
+    words = np.ascontiguousarray(bits_row, dtype=np.uint32)
+    return np.unpackbits(words.view(np.uint8), bitorder="little")[:count]
+
+
+def export_butterfly(bits: np.ndarray, log2n: int) -> np.ndarray:
+    """The settings of one permutation, (2n-1, W) words, re-indexed for the network drawn
+    in place (data never moves between stages; stage row r pairs positions that differ in
+    bit i, i = r up to the middle and 2n-2-r after it; pair p = the position with bit i
+    taken out).  Done by pushing position labels through the wiring of the recursive
+    network with every switch straight: the two labels that meet in a switch are the two
+    in-place positions that switch acts on (they must differ in exactly bit i)."""
+    n, N = log2n, 1 << log2n
+    W = stage_words(n)
+    bits = np.ascontiguousarray(bits, dtype=np.uint32).reshape(2 * n - 1, W)
+    out_bits = np.zeros((2 * n - 1, N // 2 if N >= 2 else 1), dtype=np.uint8)
+    label = np.arange(N, dtype=np.int64)          # label[q] = in-place position of what sits at q
+    per_level = []
+    for level in range(n):                        # input side, then the middle (level n-1)
+        a, b = label[0::2], label[1::2]           # switch w takes positions 2w, 2w+1 of the flat array
+        assert np.array_equal(a ^ b, np.full(N // 2, 1 << level)) and not (a & (1 << level)).any()
+        pair = ((a >> (level + 1)) << level) | (a & ((1 << level) - 1))
+        out_bits[level, pair] = _stage_bits(bits[level], N // 2)
+        per_level.append(pair)
+        if level < n - 1:                         # wiring: switch s of a block -> position s of each half
+            M = N >> level
+            blk = label.reshape(-1, M)
+            label = np.concatenate([blk[:, 0::2], blk[:, 1::2]], axis=1).reshape(-1)
+    for level in range(n - 2, -1, -1):            # output side mirrors the input side
+        out_bits[2 * n - 2 - level, per_level[level]] = _stage_bits(bits[2 * n - 2 - level], N // 2)
+    packed = np.zeros((2 * n - 1, W * 32), dtype=np.uint8)
+    packed[:, :out_bits.shape[1]] = out_bits[:, :W * 32]
+    return np.packbits(packed, axis=1, bitorder="little").view(np.uint32).reshape(2 * n - 1, W)
+
+
+def apply_butterfly(bfly: np.ndarray, x: np.ndarray, log2n: int) -> np.ndarray:
+    """Run the in-place network on a copy of x: row r swaps x[u] and x[u | 2^i] where bit p is set."""
+    n, N = log2n, 1 << log2n
+    W = stage_words(n)
+    bfly = np.ascontiguousarray(bfly, dtype=np.uint32).reshape(2 * n - 1, W)
+    y = np.array(x, copy=True)
+    for r in range(2 * n - 1):
+        i = r if r <= n - 1 else 2 * n - 2 - r
+        p = np.nonzero(_stage_bits(bfly[r], N // 2))[0].astype(np.int64)
+        u = ((p >> i) << (i + 1)) | (p & ((1 << i) - 1))
+        v = u | (1 << i)
+        y[u], y[v] = y[v].copy(), y[u].copy()
+    return y

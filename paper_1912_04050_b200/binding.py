@@ -31,6 +31,7 @@ SYMBOLS = {
     "benes_apply": (_i, [_vp, _vp, _vp, _i, _i, _vp]),
     "benes_apply_ex": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp]),
     "benes_apply_static": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp]),
+    "benes_export_butterfly": (_i, [_vp, _vp, _i, _i, _vp]),
     "benes_padded_log2n": (_i, [_sz]),
     "benes_route_padded": (_i, [_vp, _sz, _i, _vp, _vp]),
     "benes_apply_padded": (_i, [_vp, _vp, _vp, _i, _sz, _i, _vp]),
@@ -146,6 +147,13 @@ def benes_apply_static(switch_bits: torch.Tensor, inp: torch.Tensor, out: torch.
     _check(load().benes_apply_static(_dev_ptr(switch_bits, "switch_bits"), _dev_ptr(inp, "in"),
                                      _dev_ptr(out, "out"), elem_bytes, log2n, batch, _stream(stream)),
            "benes_apply_static")
+
+
+def benes_export_butterfly(switch_bits: torch.Tensor, butterfly_bits: torch.Tensor, log2n: int, batch: int,
+                           stream=None) -> None:
+    _check(load().benes_export_butterfly(_dev_ptr(switch_bits, "switch_bits"),
+                                         _dev_ptr(butterfly_bits, "butterfly_bits"), log2n, batch,
+                                         _stream(stream)), "benes_export_butterfly")
 
 
 def benes_padded_log2n(n_elems: int) -> int:

@@ -275,6 +275,14 @@ int benes_apply(const uint32_t *switch_bits, const void *in, void *out, int log2
     return benes_apply_ex(switch_bits, in, out, 4, log2n, batch, stream);
 }
 
+int benes_export_butterfly(const uint32_t *switch_bits, uint32_t *butterfly_bits, int log2n, int batch,
+                           benes_stream_t stream) {
+    if (!switch_bits || !butterfly_bits || switch_bits == butterfly_bits || bad_shape(log2n, batch))
+        return BENES_ERR_BADARG;
+    return launch_export_butterfly(switch_bits, butterfly_bits, log2n, size_t(batch),
+                                   reinterpret_cast<cudaStream_t>(stream));
+}
+
 int benes_padded_log2n(size_t n_elems) {
     if (n_elems < 1 || n_elems > (size_t(1) << BENES_MAX_LOG2N)) return 0;
     int n = 1;

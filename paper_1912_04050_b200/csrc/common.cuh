@@ -142,6 +142,8 @@ int launch_pad_perm(const uint32_t *src, uint32_t *dst, size_t n_elems, int log2
 int launch_pad_rows(const void *src, void *dst, int elem_bytes, bool pad, size_t n_elems, int log2n,
                     size_t batch, cudaStream_t s);
 
+int launch_export_butterfly(const uint32_t *bits, uint32_t *out, int log2n, size_t batch, cudaStream_t s);
+
 // ---- validation (route_levels.cu) -------------------------------------------
 int launch_validate(const uint32_t *perm, size_t total, int log2n, uint32_t *seen_words,
                     uint32_t *flag, cudaStream_t s);

@@ -73,3 +73,54 @@ int launch_pad_rows(const void *src, void *dst, int elem_bytes, bool pad, size_t
 }
 
 }  // namespace benes
+
+// ---- in-place ("butterfly") form of the switch settings ------------------------
+//
+// The same network drawn without wires between stages: data stays in place,
+// stage row r pairs positions u and u | 2^i that differ in bit i (i = r for the
+// n rows up to the middle, i = 2n-2-r after it) and a set bit swaps them.
+// Position u then holds, in its low bits, the outputs the element took at the
+// earlier stages, so the switch of the recursive layout that acts on the pair is
+//     (low i bits of u, reversed) << (n-1-i)  +  (u >> (i+1)).
+// Pair p of row r (u with bit i removed) is bit p of the row, same packing.
+namespace benes {
+namespace {
+
+__global__ void __launch_bounds__(256)
+k_export_butterfly(const uint32_t *__restrict__ bits, uint32_t *__restrict__ out, int n, size_t rows,
+                   uint32_t words_per_row) {
+    const uint32_t half = 1u << (n - 1);                       // switches per row
+    const size_t lanes_per_row = size_t(words_per_row) * 32;
+    const size_t total = rows * lanes_per_row;
+    const size_t stride = size_t(gridDim.x) * blockDim.x;
+    for (size_t idx = size_t(blockIdx.x) * blockDim.x + threadIdx.x; idx < total; idx += stride) {
+        const size_t row = idx / lanes_per_row;                // permutation * (2n-1) + stage row
+        const uint32_t p = uint32_t(idx - row * lanes_per_row);
+        const int r = int(row % size_t(2 * n - 1));
+        const int i = r <= n - 1 ? r : 2 * n - 2 - r;
+        uint32_t bit = 0;
+        if (p < half) {
+            const uint32_t lowmask = (1u << i) - 1u;
+            const uint32_t low = p & lowmask, high = p >> i;   // u = high << (i+1) | low
+            const uint32_t rev = i ? (__brev(low) >> (32 - i)) : 0u;
+            const uint32_t sw = (rev << (n - 1 - i)) + high;
+            bit = (__ldg(bits + row * words_per_row + (sw >> 5)) >> (sw & 31u)) & 1u;
+        }
+        const uint32_t word = __ballot_sync(0xFFFFFFFFu, bit);
+        if ((threadIdx.x & 31) == 0) out[row * words_per_row + (p >> 5)] = word;
+    }
+}
+
+}  // namespace
+
+int launch_export_butterfly(const uint32_t *bits, uint32_t *out, int log2n, size_t batch, cudaStream_t s) {
+    const uint32_t words = log2n >= 6 ? (1u << (log2n - 6)) : 1u;
+    const size_t rows = batch * size_t(2 * log2n - 1);
+    const size_t total = rows * words * 32;
+    size_t blocks = (total + 255) / 256;
+    if (blocks > size_t(kSMs) * 16) blocks = size_t(kSMs) * 16;
+    k_export_butterfly<<<unsigned(blocks), 256, 0, s>>>(bits, out, log2n, rows, words);
+    return launch_status();
+}
+
+}  // namespace benes

@@ -361,3 +361,31 @@ def test_bit_linear_permutations_have_short_loops():
         p = inputs.structured_perms(10)[kind].tolist()
         root, _ = loops_min_index(p)
         assert max(np.bincount(root)) <= 4
+
+
+# ---- the in-place ("butterfly") form of the settings -------------------------------------
+def test_butterfly_form_routes_every_small_permutation():
+    """The re-indexed settings, run as an in-place network (swap x[u], x[u | 2^i] where the
+    bit is set; no movement between stages), realise the permutation: all of N = 2, 4, 8."""
+    import itertools
+    for n in (1, 2, 3):
+        x = np.arange(1 << n) * 7 + 3
+        for p in itertools.permutations(range(1 << n)):
+            perm = np.array(p, dtype=np.uint32)
+            bf = oracle.export_butterfly(oracle.route(perm, n), n)
+            assert np.array_equal(oracle.apply_butterfly(bf, x, n), x[perm]), p
+
+
+@pytest.mark.parametrize("n", [4, 5, 6, 7, 9, 12])
+def test_butterfly_form_random(n):
+    perm = inputs.random_perm(n, 50 + n)
+    bits = oracle.route(perm, n)
+    bf = oracle.export_butterfly(bits, n)
+    x = np.arange(1 << n, dtype=np.uint64) * 11 + 1
+    assert np.array_equal(oracle.apply_butterfly(bf, x, n), x[perm])
+    # a re-indexing: every stage keeps its number of crossed switches
+    for r in range(2 * n - 1):
+        assert int(np.unpackbits(bf[r].view(np.uint8)).sum()) == int(np.unpackbits(bits[r].view(np.uint8)).sum())
+    # identity: nothing crossed in either form
+    ident = inputs.identity_perm(n)
+    assert not oracle.export_butterfly(oracle.route(ident, n), n).any()

@@ -250,6 +250,21 @@ def test_route_many_seeds_and_repeats(n):
             assert np.array_equal(gpu_route(perm, n), want), (n, seed)
 
 
+@pytest.mark.parametrize("n,batch", [(1, 3), (2, 5), (3, 7), (5, 4), (6, 3), (7, 2), (10, 3), (13, 2), (16, 2), (20, 1)])
+def test_export_butterfly(n, batch):
+    """The in-place form of the settings, against the oracle's re-indexing (bit-exact)."""
+    perm = inputs.random_perm_batch(n, batch, seed0=11 * n)
+    bits = oracle.route(perm, n)
+    out = torch.full((binding.benes_switch_words(n, batch),), -1, dtype=torch.int32, device="cuda")
+    binding.benes_export_butterfly(dev(bits), out, n, batch)
+    torch.cuda.synchronize()
+    got = host(out, np.uint32).reshape(bits.shape)
+    for b in range(batch):
+        assert np.array_equal(got[b], oracle.export_butterfly(bits[b], n)), b
+    x = np.arange(1 << n, dtype=np.uint64) * 3 + 1
+    assert np.array_equal(oracle.apply_butterfly(got[0], x, n), x[perm[0]])
+
+
 def test_route_batch_in_chunks():
     """A batch larger than the chunk limit is routed chunk by chunk (whole
     permutations per chunk) with a workspace sized for one chunk."""
