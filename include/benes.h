@@ -142,7 +142,11 @@ int benes_apply_static(const uint32_t *switch_bits, const void *in, void *out, i
 /*
  * Host-buffer variants: copy the inputs to the device, run, copy the result
  * back and SYNCHRONISE `stream` before returning.  Buffers are ordinary or
- * pinned host memory.  Device staging lives in the library workspace.
+ * pinned host memory (pinned memory lets the copies overlap the kernels).
+ * Device staging lives in the library workspace.  benes_route_host overlaps
+ * its copies with the computation on a second stream the library owns (one per
+ * device, created on the first call): the permutation arrives in pieces, and
+ * the stages a level has finished go back while the next levels run.
  */
 int benes_route_host(const uint32_t *perm_host, int log2n, int batch, uint32_t *switch_bits_host,
                      benes_stream_t stream);

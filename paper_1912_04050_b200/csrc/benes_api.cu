@@ -92,8 +92,32 @@ size_t apply_ws_bytes(int elem_bytes, int log2n, size_t batch) {
     return align_up((batch << log2n) * size_t(elem_bytes));
 }
 
+// Host-buffer calls overlap their copies with the computation: the permutation
+// arrives in pieces on a side stream (the bucketing pass of level 0 starts on a
+// piece as soon as it is there), and the two stages a level has finished are
+// copied to the host on the side stream while the next levels run.
+constexpr int kMaxPieces = 8;
+struct HostPipe {
+    uint32_t *bits_host = nullptr;     // finished stages go here (same layout as `bits`)
+    cudaStream_t side = nullptr;
+    int pieces = 0;                    // the permutation arrives in this many equal pieces
+    cudaEvent_t piece_ready[kMaxPieces] = {};
+    cudaEvent_t stage_ready[kMaxLevels] = {};
+};
+
+// rows `stage` of every permutation of the chunk, device -> host
+int copy_stage_rows(const HostPipe &hp, const uint32_t *bits, int n, size_t batch, int stage, int rows,
+                    cudaStream_t st) {
+    const size_t w = stage_words(n) * 4, pitch = size_t(2 * n - 1) * w;
+    BENES_CUDA_TRY(cudaMemcpy2DAsync(reinterpret_cast<char *>(hp.bits_host) + size_t(stage) * w, pitch,
+                                     reinterpret_cast<const char *>(bits) + size_t(stage) * w, pitch,
+                                     w * size_t(rows), batch, cudaMemcpyDeviceToHost, st));
+    return BENES_OK;
+}
+
 // Levels 0 .. n-kFusedLog2M-1 in HBM, then the fused tail.
-int route_levels(const uint32_t *perm, int n, size_t batch, uint32_t *bits, char *ws, cudaStream_t s) {
+int route_levels(const uint32_t *perm, int n, size_t batch, uint32_t *bits, char *ws, cudaStream_t s,
+                 const HostPipe *hp = nullptr) {
     const size_t T = batch << n;
     uint4 *Sbuf[2];
     uint32_t *Qbuf[2];
@@ -123,11 +147,24 @@ int route_levels(const uint32_t *perm, int n, size_t batch, uint32_t *bits, char
         ProfileScope ps(kInverse, s);
         // the 64-bit word array is free until the first level is labelled
         // (the bucketed form needs whole buckets of 2^18 entries)
-        if (g_inverse_partitioned && T >= (size_t(1) << kInversePartitionMinLog2) &&
-            (T & ((size_t(1) << 18) - 1)) == 0)
-            rc = launch_inverse_partitioned(perm, Sbuf[0], Qbuf[0], Wd, fill, T, n, s);
-        else
-            rc = launch_inverse(perm, Sbuf[0], Qbuf[0], T, n, s);
+        const bool bucketed = g_inverse_partitioned && T >= (size_t(1) << kInversePartitionMinLog2) &&
+                              (T & ((size_t(1) << 18) - 1)) == 0;
+        const int pieces = hp ? hp->pieces : 0;
+        if (bucketed && pieces > 1) {
+            if ((rc = launch_inverse_clear(fill, T, s))) return rc;
+            const size_t per = T / size_t(pieces);
+            for (int i = 0; i < pieces; ++i) {
+                BENES_CUDA_TRY(cudaStreamWaitEvent(s, hp->piece_ready[i], 0));
+                if ((rc = launch_inverse_partition_piece(perm, Sbuf[0], Wd, fill, T, per * size_t(i), per,
+                                                         n, s)))
+                    return rc;
+            }
+            rc = launch_inverse_scatter(Wd, Qbuf[0], T, n, s);
+        } else {
+            for (int i = 0; i < pieces; ++i) BENES_CUDA_TRY(cudaStreamWaitEvent(s, hp->piece_ready[i], 0));
+            rc = bucketed ? launch_inverse_partitioned(perm, Sbuf[0], Qbuf[0], Wd, fill, T, n, s)
+                          : launch_inverse(perm, Sbuf[0], Qbuf[0], T, n, s);
+        }
         if (rc) return rc;
     }
     int cur = 0;
@@ -156,9 +193,43 @@ int route_levels(const uint32_t *perm, int n, size_t batch, uint32_t *bits, char
                 return rc;
         }
         cur ^= 1;
+        if (hp && hp->bits_host) {
+            // stages `level` and `out_stage` are final: send them home behind the computation
+            BENES_CUDA_TRY(cudaEventRecord(hp->stage_ready[level], s));
+            BENES_CUDA_TRY(cudaStreamWaitEvent(hp->side, hp->stage_ready[level], 0));
+            if ((rc = copy_stage_rows(*hp, bits, n, batch, level, 1, hp->side))) return rc;
+            if ((rc = copy_stage_rows(*hp, bits, n, batch, out_stage, 1, hp->side))) return rc;
+        }
     }
-    ProfileScope ps(kFused, s);
-    return launch_fused(Sbuf[cur], 1, T, kFusedLog2M, bits, n, s);
+    {
+        ProfileScope ps(kFused, s);
+        if ((rc = launch_fused(Sbuf[cur], 1, T, kFusedLog2M, bits, n, s))) return rc;
+    }
+    if (hp && hp->bits_host) {
+        // the stages of the in-CTA levels are one run of rows in the middle
+        const int first = n - kFusedLog2M;
+        if ((rc = copy_stage_rows(*hp, bits, n, batch, first, 2 * kFusedLog2M - 1, s))) return rc;
+    }
+    return BENES_OK;
+}
+
+// Side stream and events of the host-buffer calls, one set per device.
+int host_pipe_for_current_device(HostPipe **out) {
+    static HostPipe pipes[kMaxDevices];
+    static bool ready[kMaxDevices] = {};
+    int dev = 0;
+    BENES_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return BENES_ERR_CUDA;
+    std::lock_guard<std::mutex> lk(g_mu);
+    HostPipe &hp = pipes[dev];
+    if (!ready[dev]) {
+        BENES_CUDA_TRY(cudaStreamCreateWithFlags(&hp.side, cudaStreamNonBlocking));
+        for (cudaEvent_t &e : hp.piece_ready) BENES_CUDA_TRY(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+        for (cudaEvent_t &e : hp.stage_ready) BENES_CUDA_TRY(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+        ready[dev] = true;
+    }
+    *out = &hp;
+    return BENES_OK;
 }
 
 }  // namespace
@@ -336,6 +407,29 @@ int benes_route_host(const uint32_t *perm_host, int log2n, int batch, uint32_t *
     char *base = static_cast<char *>(ws);
     uint32_t *d_perm = reinterpret_cast<uint32_t *>(base + align_up(inner));
     uint32_t *d_bits = reinterpret_cast<uint32_t *>(base + align_up(inner) + align_up(perm_bytes));
+    const int n = log2n;
+    if (n > kFusedLog2M && level_chunk(n, size_t(batch)) == size_t(batch)) {
+        // one chunk: copies overlapped with the levels (see HostPipe)
+        HostPipe *hp = nullptr;
+        if ((rc = host_pipe_for_current_device(&hp))) return rc;
+        const size_t T = size_t(batch) << n;
+        hp->bits_host = switch_bits_host;
+        hp->pieces = (T >= (size_t(1) << 23)) ? kMaxPieces : 1;
+        // the side stream must not touch the workspace before earlier work on `s` is done
+        BENES_CUDA_TRY(cudaEventRecord(hp->stage_ready[kMaxLevels - 1], s));
+        BENES_CUDA_TRY(cudaStreamWaitEvent(hp->side, hp->stage_ready[kMaxLevels - 1], 0));
+        const size_t per = perm_bytes / size_t(hp->pieces);
+        for (int i = 0; i < hp->pieces; ++i) {
+            BENES_CUDA_TRY(cudaMemcpyAsync(reinterpret_cast<char *>(d_perm) + per * size_t(i),
+                                           reinterpret_cast<const char *>(perm_host) + per * size_t(i), per,
+                                           cudaMemcpyHostToDevice, hp->side));
+            BENES_CUDA_TRY(cudaEventRecord(hp->piece_ready[i], hp->side));
+        }
+        rc = route_levels(d_perm, n, size_t(batch), d_bits, base, s, hp);
+        cudaError_t e1 = cudaStreamSynchronize(hp->side), e2 = cudaStreamSynchronize(s);
+        if (rc) return rc;
+        return (e1 == cudaSuccess && e2 == cudaSuccess) ? BENES_OK : BENES_ERR_CUDA;
+    }
     BENES_CUDA_TRY(cudaMemcpyAsync(d_perm, perm_host, perm_bytes, cudaMemcpyHostToDevice, s));
     rc = benes_route(d_perm, log2n, batch, d_bits, stream);
     if (rc) return rc;

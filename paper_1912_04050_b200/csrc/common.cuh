@@ -90,6 +90,11 @@ constexpr int kInversePartitionMinLog2 = 22;
 constexpr int kInverseMaxBuckets = 4096;
 int launch_inverse_partitioned(const uint32_t *perm, uint4 *S, uint32_t *Q, void *pairs, uint32_t *fill,
                                size_t total, int log2m, cudaStream_t s);
+int launch_inverse_clear(uint32_t *fill, size_t total, cudaStream_t s);
+int launch_inverse_partition_piece(const uint32_t *perm, uint4 *S, void *pairs, uint32_t *fill,
+                                   size_t total, size_t j_first, size_t count, int log2m,
+                                   cudaStream_t s);
+int launch_inverse_scatter(const void *pairs, uint32_t *Q, size_t total, int log2m, cudaStream_t s);
 // Pointer jumping over all outputs (successor build, log2m-2 in-place passes,
 // last pass + output-side bits) in ONE cooperative launch; `gate` (may be
 // null) is a device word: the kernel returns at once while it is 0.

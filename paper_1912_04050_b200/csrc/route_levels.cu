@@ -73,12 +73,12 @@ constexpr int kPartThreads = 1024;
 
 __global__ void __launch_bounds__(kPartThreads)
 k_inverse_partition(const uint32_t *__restrict__ P, uint4 *__restrict__ S, uint2 *__restrict__ pairs,
-                    uint32_t *__restrict__ fill, uint32_t buckets, uint32_t mmask) {
+                    uint32_t *__restrict__ fill, uint32_t buckets, uint32_t mmask, size_t j_first) {
     extern __shared__ uint32_t sh[];           // count[buckets], then offset[buckets]
     uint32_t *count = sh, *offset = sh + buckets;
     for (uint32_t b = threadIdx.x; b < buckets; b += kPartThreads) count[b] = 0u;
     __syncthreads();
-    const size_t j0 = size_t(blockIdx.x) * kPartChunk;
+    const size_t j0 = j_first + size_t(blockIdx.x) * kPartChunk;
     constexpr int kPer = kPartChunk / kPartThreads;
     uint32_t dest[kPer], rank[kPer];
 #pragma unroll
@@ -258,18 +258,34 @@ int cooperative_grid(int *out) {
 
 }  // namespace
 
+// Pass 1 over elements [j_first, j_first + count) (a multiple of 8192); `fill`
+// must have been cleared before the first piece.  Pass 2 over everything.
+int launch_inverse_clear(uint32_t *fill, size_t total, cudaStream_t s) {
+    BENES_CUDA_TRY(cudaMemsetAsync(fill, 0, (total >> kBucketLog2) * 4, s));
+    return BENES_OK;
+}
+
+int launch_inverse_partition_piece(const uint32_t *perm, uint4 *S, void *pairs, uint32_t *fill,
+                                   size_t total, size_t j_first, size_t count, int log2m,
+                                   cudaStream_t s) {
+    const uint32_t buckets = uint32_t(total >> kBucketLog2);
+    k_inverse_partition<<<unsigned(count / kPartChunk), kPartThreads, size_t(buckets) * 8, s>>>(
+        perm, S, static_cast<uint2 *>(pairs), fill, buckets, (1u << log2m) - 1u, j_first);
+    return launch_status();
+}
+
+int launch_inverse_scatter(const void *pairs, uint32_t *Q, size_t total, int log2m, cudaStream_t s) {
+    k_inverse_scatter<<<unsigned((total + kThreads - 1) / kThreads), kThreads, 0, s>>>(
+        static_cast<const uint2 *>(pairs), Q, total, (1u << log2m) - 1u);
+    return launch_status();
+}
+
 int launch_inverse_partitioned(const uint32_t *perm, uint4 *S, uint32_t *Q, void *pairs, uint32_t *fill,
                                size_t total, int log2m, cudaStream_t s) {
-    const uint32_t buckets = uint32_t(total >> kBucketLog2);
-    const uint32_t mmask = (1u << log2m) - 1u;
-    BENES_CUDA_TRY(cudaMemsetAsync(fill, 0, size_t(buckets) * 4, s));
-    k_inverse_partition<<<unsigned(total / kPartChunk), kPartThreads, size_t(buckets) * 8, s>>>(
-        perm, S, static_cast<uint2 *>(pairs), fill, buckets, mmask);
-    int rc = launch_status();
-    if (rc) return rc;
-    k_inverse_scatter<<<unsigned((total + kThreads - 1) / kThreads), kThreads, 0, s>>>(
-        static_cast<const uint2 *>(pairs), Q, total, mmask);
-    return launch_status();
+    int rc;
+    if ((rc = launch_inverse_clear(fill, total, s))) return rc;
+    if ((rc = launch_inverse_partition_piece(perm, S, pairs, fill, total, 0, total, log2m, s))) return rc;
+    return launch_inverse_scatter(pairs, Q, total, log2m, s);
 }
 
 int launch_inverse(const uint32_t *perm, uint4 *S, uint32_t *Q, size_t total, int log2m,

@@ -310,16 +310,28 @@ def test_route_n2p28_properties():
 
 
 # ---- host-buffer entry points, validation, robustness -------------------------------------------
-def test_host_entry_points():
-    n, batch = 15, 2
+@pytest.mark.parametrize("n,batch,pinned", [(15, 2, False), (17, 3, False), (18, 1, True), (23, 1, True), (23, 1, False)])
+def test_host_entry_points(n, batch, pinned):
+    """Host buffers in and out; above the in-CTA size the copies are overlapped with
+    the levels (the permutation arrives in pieces from N = 2^23 on)."""
     perm = inputs.random_perm_batch(n, batch, seed0=5)
-    bits = np.empty((batch, 2 * n - 1, (1 << n) // 64), dtype=np.uint32)
-    binding.benes_route_host(perm, n, batch, bits)
+    bits = np.full((batch, 2 * n - 1, (1 << n) // 64), 0xAAAAAAAA, dtype=np.uint32)
+    if pinned:
+        perm_t = torch.from_numpy(perm.view(np.int32)).pin_memory()
+        bits_t = torch.from_numpy(bits.view(np.int32)).pin_memory()
+        binding.benes_route_host(perm_t, n, batch, bits_t)
+        bits = bits_t.numpy().view(np.uint32)
+    else:
+        binding.benes_route_host(perm, n, batch, bits)
     assert np.array_equal(bits, oracle.route(perm, n))
     x = inputs.payload_u64(batch << n, 4).reshape(batch, -1)
     out = np.empty_like(x)
     binding.benes_apply_host(bits, x, out, 8, n, batch)
     assert np.array_equal(out, np.take_along_axis(x, perm.astype(np.int64), axis=1))
+    # a second call right away reuses the side stream and the workspace
+    bits2 = np.zeros_like(bits)
+    binding.benes_route_host(perm, n, batch, bits2)
+    assert np.array_equal(bits2, bits)
 
 
 def test_caller_workspace_is_used_and_checked():
