@@ -29,9 +29,11 @@ extern unsigned long long g_launches;
         if (e_ != cudaSuccess) return BENES_ERR_CUDA;          \
     } while (0)
 
+// Result of the launch just issued; a launch error is taken off the runtime's
+// error state so that it is reported once, by the call that caused it.
 inline int launch_status() {
     ++g_launches;
-    return cudaPeekAtLastError() == cudaSuccess ? BENES_OK : BENES_ERR_CUDA;
+    return cudaGetLastError() == cudaSuccess ? BENES_OK : BENES_ERR_CUDA;
 }
 
 // Optional event timing of a group of launches of one kind (see benes.h).
