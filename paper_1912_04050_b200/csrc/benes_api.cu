@@ -119,11 +119,11 @@ int copy_stage_rows(const HostPipe &hp, const uint32_t *bits, int n, size_t batc
 int route_levels(const uint32_t *perm, int n, size_t batch, uint32_t *bits, char *ws, cudaStream_t s,
                  const HostPipe *hp = nullptr) {
     const size_t T = batch << n;
-    uint4 *Sbuf[2];
+    void *Sbuf[2];                     // two generations of switch records (wide: 16 B per switch)
     uint32_t *Qbuf[2];
     size_t off = 0;
-    Sbuf[0] = reinterpret_cast<uint4 *>(ws + off); off += align_up(T * 8);
-    Sbuf[1] = reinterpret_cast<uint4 *>(ws + off); off += align_up(T * 8);
+    Sbuf[0] = ws + off; off += align_up(T * 8);
+    Sbuf[1] = ws + off; off += align_up(T * 8);
     Qbuf[0] = reinterpret_cast<uint32_t *>(ws + off); off += align_up(T * 4);
     Qbuf[1] = reinterpret_cast<uint32_t *>(ws + off); off += align_up(T * 4);
     unsigned long long *Wd = reinterpret_cast<unsigned long long *>(ws + off); off += align_up(T * 8);
@@ -150,20 +150,21 @@ int route_levels(const uint32_t *perm, int n, size_t batch, uint32_t *bits, char
         const bool bucketed = g_inverse_partitioned && T >= (size_t(1) << kInversePartitionMinLog2) &&
                               (T & ((size_t(1) << 18) - 1)) == 0;
         const int pieces = hp ? hp->pieces : 0;
+        const bool pk = rec_is_packed(n, kappa);
         if (bucketed && pieces > 1) {
             if ((rc = launch_inverse_clear(fill, T, s))) return rc;
             const size_t per = T / size_t(pieces);
             for (int i = 0; i < pieces; ++i) {
                 BENES_CUDA_TRY(cudaStreamWaitEvent(s, hp->piece_ready[i], 0));
-                if ((rc = launch_inverse_partition_piece(perm, Sbuf[0], Wd, fill, T, per * size_t(i), per,
-                                                         n, s)))
+                if ((rc = launch_inverse_partition_piece(perm, Sbuf[0], pk, Wd, fill, T, per * size_t(i),
+                                                         per, n, s)))
                     return rc;
             }
             rc = launch_inverse_scatter(Wd, Qbuf[0], T, n, s);
         } else {
             for (int i = 0; i < pieces; ++i) BENES_CUDA_TRY(cudaStreamWaitEvent(s, hp->piece_ready[i], 0));
-            rc = bucketed ? launch_inverse_partitioned(perm, Sbuf[0], Qbuf[0], Wd, fill, T, n, s)
-                          : launch_inverse(perm, Sbuf[0], Qbuf[0], T, n, s);
+            rc = bucketed ? launch_inverse_partitioned(perm, Sbuf[0], pk, Qbuf[0], Wd, fill, T, n, s)
+                          : launch_inverse(perm, Sbuf[0], pk, Qbuf[0], T, n, s);
         }
         if (rc) return rc;
     }
@@ -171,25 +172,26 @@ int route_levels(const uint32_t *perm, int n, size_t batch, uint32_t *bits, char
     for (int level = 0; n - level > kFusedLog2M; ++level) {
         const int m = n - level;
         const int out_stage = 2 * n - 2 - level;
-        uint4 *S = Sbuf[cur];
+        void *S = Sbuf[cur];
         uint32_t *Q = Qbuf[cur];
+        const bool pk = rec_is_packed(m, kappa), pk_next = rec_is_packed(m - 1, kappa);
         uint32_t *gate = nullptr;
         if (kappa) {
             // ruler-sampled labelling; raises `gate` if a walk had to give up
             gate = gates + level;
-            if ((rc = sampled_label(S, Q, Sbuf[cur ^ 1], sc, T, m, kappa, uint32_t(level), cap, L, out_stage,
-                                    gate, s)))
+            if ((rc = sampled_label(S, pk, Q, Sbuf[cur ^ 1], pk_next, sc, T, m, kappa, uint32_t(level), cap, L,
+                                    out_stage, gate, s)))
                 return rc;
         }
         // pointer jumping over all outputs: the whole labelling when sampling is
         // off, otherwise gated (returns at once unless this level's walks gave up)
         {
             ProfileScope ps(kFullLabel, s);
-            if ((rc = launch_full_label(S, Q, Wd, T, m, L, out_stage, gate, s))) return rc;
+            if ((rc = launch_full_label(S, pk, Q, Wd, T, m, L, out_stage, gate, s))) return rc;
         }
         {
             ProfileScope ps(kSplit, s);
-            if ((rc = launch_split(S, Q, Sbuf[cur ^ 1], Qbuf[cur ^ 1], T, m, L, level, out_stage, gate, s)))
+            if ((rc = launch_split(S, pk, Q, Sbuf[cur ^ 1], pk_next, Qbuf[cur ^ 1], T, m, L, level, out_stage, gate, s)))
                 return rc;
         }
         cur ^= 1;
@@ -203,7 +205,7 @@ int route_levels(const uint32_t *perm, int n, size_t batch, uint32_t *bits, char
     }
     {
         ProfileScope ps(kFused, s);
-        if ((rc = launch_fused(Sbuf[cur], 1, T, kFusedLog2M, bits, n, s))) return rc;
+        if ((rc = launch_fused(Sbuf[cur], rec_is_packed(kFusedLog2M, kappa) ? 2 : 1, T, kFusedLog2M, bits, n, s))) return rc;
     }
     if (hp && hp->bits_host) {
         // the stages of the in-CTA levels are one run of rows in the middle

@@ -65,15 +65,59 @@ struct BitsLayout {
 };
 
 // ---- layout of a level in HBM ------------------------------------------------
-// A level of the per-level path keeps its sub-permutations as one 16-byte
-// record per output switch t of the flat array,
-//     S[t] = { P[2t], P[2t+1], owner, 0 },
-// P block-local, and the inverses Q as a plain uint32 array.  `owner` is
-// kUnowned until a walk of the sampled labelling claims the switch; it sits in
-// the record so that claiming costs no memory access of its own (the walker
-// has just fetched the record for P).
-__device__ __forceinline__ uint32_t rec_p(const uint4 *S, uint32_t j) {
-    return reinterpret_cast<const uint32_t *>(S)[(size_t(j >> 1) << 2) | (j & 1u)];
+// A level of the per-level path keeps its sub-permutations as one record per
+// output switch t of the flat array, and the inverses Q as a plain uint32
+// array (read at random, never claimed).  Two record formats:
+//
+//   wide   (16 B)  { P[2t], P[2t+1], owner, 0 }, P block-local; owner is
+//                  kUnowned until a walk of the sampled labelling claims the
+//                  switch with a compare-and-swap.  It sits in the record so
+//                  that claiming hits the sector the walker has just fetched.
+//   packed (8 B)   P[2t] | P[2t+1] << m | owner << 2m for blocks of 2^m outputs,
+//                  owner local to the block, all ones = unowned.  One 64-bit
+//                  atomic AND both returns the two P values and claims the
+//                  switch, i.e. one memory operation instead of two.  Used
+//                  when the owner fits with room for the all-ones value:
+//                  2m + (m - kappa + 1) < 64.
+//
+// Owner = (ruler output that claimed the switch) << 1 | side of arrival.
+__host__ __device__ inline bool rec_is_packed(int m, int kappa) {
+    return kappa != 0 && 3 * m - kappa + 1 < 64;
+}
+
+template <bool PACKED>
+__device__ __forceinline__ void rec_read(const void *S, size_t t, int m, uint32_t &p0, uint32_t &p1) {
+    if (PACKED) {
+        const unsigned long long w = __ldcs(static_cast<const unsigned long long *>(S) + t);
+        const uint32_t mask = (1u << m) - 1u;
+        p0 = uint32_t(w) & mask;
+        p1 = uint32_t(w >> m) & mask;
+    } else {
+        const uint4 r = __ldcs(static_cast<const uint4 *>(S) + t);
+        const uint32_t mask = (1u << m) - 1u;
+        p0 = r.x & mask;
+        p1 = r.y & mask;
+    }
+}
+
+// one P value, P[j], read at random
+template <bool PACKED>
+__device__ __forceinline__ uint32_t rec_p(const void *S, uint32_t j, int m) {
+    if (PACKED) {
+        const unsigned long long w = __ldg(static_cast<const unsigned long long *>(S) + (j >> 1));
+        return uint32_t(w >> ((j & 1u) ? m : 0)) & ((1u << m) - 1u);
+    }
+    return static_cast<const uint32_t *>(S)[(size_t(j >> 1) << 2) | (j & 1u)] & ((1u << m) - 1u);
+}
+
+// an unowned record of a level with blocks of 2^m outputs
+template <bool PACKED>
+__device__ __forceinline__ void rec_write(void *S, size_t t, int m, uint32_t p0, uint32_t p1) {
+    if (PACKED)
+        static_cast<unsigned long long *>(S)[t] =
+            (unsigned long long)p0 | ((unsigned long long)p1 << m) | (~0ull << (2 * m));
+    else
+        static_cast<uint4 *>(S)[t] = make_uint4(p0, p1, kUnowned, 0u);
 }
 
 __device__ __forceinline__ unsigned long long make_word(uint32_t nxt, uint32_t mn) {
@@ -83,30 +127,30 @@ __device__ __forceinline__ unsigned long long make_word(uint32_t nxt, uint32_t m
 // ---- per-level HBM path (route_levels.cu) ----------------------------------
 // total = batch * N flat elements (<= 2^30), all blocks of one level per launch.
 // Level 0: S records from the caller's permutation, and Q[P[j]] = j.
-int launch_inverse(const uint32_t *perm, uint4 *S, uint32_t *Q, size_t total, int log2m,
+int launch_inverse(const uint32_t *perm, void *S, bool packed, uint32_t *Q, size_t total, int log2m,
                    cudaStream_t s);
 // The same for total >= 2^kInversePartitionMinLog2 in two streaming passes:
 // `pairs` = total x 8 bytes of scratch, `fill` = total >> 18 zero-initialised
 // counters (at most kInverseMaxBuckets).
 constexpr int kInversePartitionMinLog2 = 22;
 constexpr int kInverseMaxBuckets = 4096;
-int launch_inverse_partitioned(const uint32_t *perm, uint4 *S, uint32_t *Q, void *pairs, uint32_t *fill,
-                               size_t total, int log2m, cudaStream_t s);
+int launch_inverse_partitioned(const uint32_t *perm, void *S, bool packed, uint32_t *Q, void *pairs,
+                               uint32_t *fill, size_t total, int log2m, cudaStream_t s);
 int launch_inverse_clear(uint32_t *fill, size_t total, cudaStream_t s);
-int launch_inverse_partition_piece(const uint32_t *perm, uint4 *S, void *pairs, uint32_t *fill,
+int launch_inverse_partition_piece(const uint32_t *perm, void *S, bool packed, void *pairs, uint32_t *fill,
                                    size_t total, size_t j_first, size_t count, int log2m,
                                    cudaStream_t s);
 int launch_inverse_scatter(const void *pairs, uint32_t *Q, size_t total, int log2m, cudaStream_t s);
 // Pointer jumping over all outputs (successor build, log2m-2 in-place passes,
 // last pass + output-side bits) in ONE cooperative launch; `gate` (may be
 // null) is a device word: the kernel returns at once while it is 0.
-int launch_full_label(const uint4 *S, const uint32_t *Q, unsigned long long *Wd, size_t total,
+int launch_full_label(const void *S, bool packed, const uint32_t *Q, unsigned long long *Wd, size_t total,
                       int log2m, BitsLayout L, int out_stage, const uint32_t *gate, cudaStream_t s);
 // Input-side bits + next level's inverses; also the next level's records
 // (owner reset) if `gate` is null or *gate != 0 (otherwise the colouring kernel
 // of the sampled labelling has written them already).
-int launch_split(const uint4 *S, const uint32_t *Q, uint4 *Sn, uint32_t *Qn, size_t total,
-                 int log2m, BitsLayout L, int in_stage, int out_stage, const uint32_t *gate,
+int launch_split(const void *S, bool packed, const uint32_t *Q, void *Sn, bool next_packed, uint32_t *Qn,
+                 size_t total, int log2m, BitsLayout L, int in_stage, int out_stage, const uint32_t *gate,
                  cudaStream_t s);
 
 // ---- ruler-sampled loop labelling (route_sampled.cu) --------------------------
@@ -120,8 +164,8 @@ void sampled_scratch_carve(char *base, size_t total, int kappa, SampledScratch *
 // Labels every loop of the level, writes the output-side stage and the next
 // level's records Sn; raises *gate if some walk exceeded `cap` hops (the level
 // must then be relabelled and Sn rewritten).
-int sampled_label(uint4 *S, const uint32_t *Q, uint4 *Sn, const SampledScratch &sc, size_t total,
-                  int log2m, int kappa, uint32_t salt, uint32_t cap, BitsLayout L, int out_stage,
+int sampled_label(void *S, bool packed, const uint32_t *Q, void *Sn, bool next_packed,
+                  const SampledScratch &sc, size_t total, int log2m, int kappa, uint32_t salt, uint32_t cap, BitsLayout L, int out_stage,
                   uint32_t *gate, cudaStream_t s);
 // owner[0] and owner[1] must be all kUnowned before the first sampled_label.
 int sampled_scratch_reset(const SampledScratch &sc, size_t total, int kappa, cudaStream_t s);
@@ -129,7 +173,7 @@ int sampled_scratch_reset(const SampledScratch &sc, size_t total, int kappa, cud
 // ---- fused path (route_fused.cu) -------------------------------------------
 // Finishes levels (n - log2m) .. n-1 of every block of size 2^log2m of the flat
 // level array (total elements), one CTA per block.  log2m <= kFusedLog2M.
-// P is a plain uint32 array if records == 0, else the 16-byte switch records.
+// P is a plain uint32 array if records == 0, wide records if 1, packed records if 2.
 int launch_fused(const void *P, int records, size_t total, int log2m, uint32_t *bits, int log2n,
                  cudaStream_t s);
 

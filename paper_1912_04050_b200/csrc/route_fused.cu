@@ -78,10 +78,17 @@ k_route_fused(const uint32_t *__restrict__ P, int records, uint32_t *__restrict_
     const size_t local_first_switch = (flat0 & (N - 1)) >> 1;
     uint32_t *my_bits = bits + perm * size_t(2 * n - 1) * stage_w + (local_first_switch >> 5);
 
-    // plain array, or 16-byte switch records {P[2t], P[2t+1], -, -}
+    // plain array (0), wide switch records {P[2t], P[2t+1], -, -} (1), or packed
+    // records P[2t] | P[2t+1] << LOGM | ... (2)
     for (int j = tid; j < M; j += T) {
         size_t f = flat0 + j;
-        uint32_t v = records ? P[((f >> 1) << 2) | (f & 1)] : P[f];
+        uint32_t v;
+        if (records == 2) {
+            const unsigned long long w = reinterpret_cast<const unsigned long long *>(P)[f >> 1];
+            v = uint32_t(w >> ((f & 1) ? LOGM : 0));
+        } else {
+            v = records ? P[((f >> 1) << 2) | (f & 1)] : P[f];
+        }
         Pa[j] = uint16_t(v & uint32_t(M - 1));
     }
     __syncthreads();

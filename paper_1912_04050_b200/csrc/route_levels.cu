@@ -38,9 +38,11 @@ inline int grid_for(size_t work_items, int per_sm = 8) {
 
 // a1 at level 0: records of two switches per thread (16-byte load of four
 // values of the caller's permutation) and Q[base + P[j]] = j - base.
+template <bool PACKED>
 __global__ void __launch_bounds__(kThreads)
-k_inverse(const uint4 *__restrict__ P4, uint4 *__restrict__ S, uint32_t *__restrict__ Q,
-          size_t quads, uint32_t mmask) {
+k_inverse(const uint4 *__restrict__ P4, void *__restrict__ S, uint32_t *__restrict__ Q,
+          size_t quads, int m) {
+    const uint32_t mmask = (1u << m) - 1u;
     size_t stride = size_t(gridDim.x) * blockDim.x;
     for (size_t i = size_t(blockIdx.x) * blockDim.x + threadIdx.x; i < quads; i += stride) {
         uint4 p = __ldcs(P4 + i);
@@ -48,8 +50,8 @@ k_inverse(const uint4 *__restrict__ P4, uint4 *__restrict__ S, uint32_t *__restr
         size_t j = i * 4;
         size_t base = j & ~size_t(mmask);
         uint32_t jl = uint32_t(j) & mmask;
-        S[2 * i] = make_uint4(p.x, p.y, kUnowned, 0u);
-        S[2 * i + 1] = make_uint4(p.z, p.w, kUnowned, 0u);
+        rec_write<PACKED>(S, 2 * i, m, p.x, p.y);
+        rec_write<PACKED>(S, 2 * i + 1, m, p.z, p.w);
         Q[base + p.x] = jl;
         Q[base + p.y] = jl + 1;
         Q[base + p.z] = jl + 2;
@@ -71,9 +73,11 @@ constexpr int kBucketLog2 = 18;
 constexpr int kPartChunk = 8192;
 constexpr int kPartThreads = 1024;
 
+template <bool PACKED>
 __global__ void __launch_bounds__(kPartThreads)
-k_inverse_partition(const uint32_t *__restrict__ P, uint4 *__restrict__ S, uint2 *__restrict__ pairs,
-                    uint32_t *__restrict__ fill, uint32_t buckets, uint32_t mmask, size_t j_first) {
+k_inverse_partition(const uint32_t *__restrict__ P, void *__restrict__ S, uint2 *__restrict__ pairs,
+                    uint32_t *__restrict__ fill, uint32_t buckets, int m, size_t j_first) {
+    const uint32_t mmask = (1u << m) - 1u;
     extern __shared__ uint32_t sh[];           // count[buckets], then offset[buckets]
     uint32_t *count = sh, *offset = sh + buckets;
     for (uint32_t b = threadIdx.x; b < buckets; b += kPartThreads) count[b] = 0u;
@@ -87,7 +91,7 @@ k_inverse_partition(const uint32_t *__restrict__ P, uint4 *__restrict__ S, uint2
         const size_t j = j0 + 2 * (size_t(i / 2) * kPartThreads + threadIdx.x);
         const uint2 p = __ldcs(reinterpret_cast<const uint2 *>(P + j));
         const uint32_t px = p.x & mmask, py = p.y & mmask;
-        S[j >> 1] = make_uint4(px, py, kUnowned, 0u);
+        rec_write<PACKED>(S, j >> 1, m, px, py);
         const uint32_t base = uint32_t(j) & ~mmask;
         dest[i] = base + px;
         dest[i + 1] = base + py;
@@ -130,11 +134,13 @@ __device__ __forceinline__ unsigned long long jump(unsigned long long w, unsigne
 //   build : W[j] = (g(j), j), g(j) = base + Q[base + (P[j^1] ^ 1)]
 //   passes: W[j] <- (W[nxt].nxt, min(mn, W[nxt].mn)), in place
 //   last  : even outputs only; colour = leader & 1 -> output-side stage word
+template <bool PACKED>
 __global__ void __launch_bounds__(kThreads)
-k_full_label(const uint4 *__restrict__ S, const uint32_t *__restrict__ Q,
-             unsigned long long *__restrict__ Wd, size_t total, uint32_t mmask, int passes,
+k_full_label(const void *__restrict__ S, const uint32_t *__restrict__ Q,
+             unsigned long long *__restrict__ Wd, size_t total, int m, int passes,
              BitsLayout L, int out_stage, const uint32_t *__restrict__ gate) {
     if (gate && *gate == 0u) return;        // same value for every thread of the grid
+    const uint32_t mmask = (1u << m) - 1u;
     cg::grid_group grid = cg::this_grid();
     const size_t stride = size_t(gridDim.x) * blockDim.x;
     const size_t first = size_t(blockIdx.x) * blockDim.x + threadIdx.x;
@@ -142,12 +148,13 @@ k_full_label(const uint4 *__restrict__ S, const uint32_t *__restrict__ Q,
 
     const size_t switches = total / 2;
     for (size_t t = first; t < switches; t += stride) {
-        uint4 r = __ldg(S + t);
+        uint32_t p0, p1;
+        rec_read<PACKED>(S, t, m, p0, p1);
         size_t j = 2 * t;
         size_t base = j & ~size_t(mmask);
         uint32_t b32 = uint32_t(base);
-        uint32_t g0 = b32 + (__ldg(Q + base + ((r.y & mmask) ^ 1u)) & mmask);
-        uint32_t g1 = b32 + (__ldg(Q + base + ((r.x & mmask) ^ 1u)) & mmask);
+        uint32_t g0 = b32 + (__ldg(Q + base + (p1 ^ 1u)) & mmask);
+        uint32_t g1 = b32 + (__ldg(Q + base + (p0 ^ 1u)) & mmask);
         ulonglong2 a;
         a.x = make_word(g0, uint32_t(j));
         a.y = make_word(g1, uint32_t(j) + 1u);
@@ -188,27 +195,29 @@ k_full_label(const uint4 *__restrict__ S, const uint32_t *__restrict__ Q,
 // position tl of the upper half-block takes P[2t or 2t+1] >> 1 of switch tl,
 // so two neighbouring threads hold the two values of one record of the next
 // level; they exchange them with a shuffle and store whole records.
+template <bool PACKED, bool NEXT_PACKED>
 __global__ void __launch_bounds__(kThreads)
-k_split(const uint4 *__restrict__ S, const uint2 *__restrict__ Q2, uint4 *__restrict__ Sn,
-        uint32_t *__restrict__ Qn, size_t switches, uint32_t mmask, BitsLayout L, int in_stage,
+k_split(const void *__restrict__ S, const uint2 *__restrict__ Q2, void *__restrict__ Sn,
+        uint32_t *__restrict__ Qn, size_t switches, int m, BitsLayout L, int in_stage,
         int out_stage, const uint32_t *__restrict__ gate) {
     const bool with_records = !gate || *gate != 0u;
+    const uint32_t mmask = (1u << m) - 1u;
     size_t stride = size_t(gridDim.x) * blockDim.x;
     const uint32_t H = (mmask + 1) >> 1;
     for (size_t t = size_t(blockIdx.x) * blockDim.x + threadIdx.x; t < switches; t += stride) {
         size_t base = (2 * t) & ~size_t(mmask);
         uint32_t tl = uint32_t(t - base / 2);
         if (with_records) {
-            uint4 r = __ldcs(S + t);
-            r.x &= mmask; r.y &= mmask;
+            uint32_t px, py;
+            rec_read<PACKED>(S, t, m, px, py);
             // colour of output 2t
             uint32_t c = (L.bits[L.word(out_stage, t >> 5)] >> (t & 31)) & 1u;
-            uint32_t up = (c ? r.y : r.x) >> 1, lo = (c ? r.x : r.y) >> 1;
+            uint32_t up = (c ? py : px) >> 1, lo = (c ? px : py) >> 1;
             uint32_t got = __shfl_xor_sync(0xFFFFFFFFu, (tl & 1u) ? up : lo, 1);
             if (tl & 1u)
-                Sn[(base >> 1) + (H >> 1) + (tl >> 1)] = make_uint4(got, lo, kUnowned, 0u);
+                rec_write<NEXT_PACKED>(Sn, (base >> 1) + (H >> 1) + (tl >> 1), m - 1, got, lo);
             else
-                Sn[(base >> 1) + (tl >> 1)] = make_uint4(up, got, kUnowned, 0u);
+                rec_write<NEXT_PACKED>(Sn, (base >> 1) + (tl >> 1), m - 1, up, got);
         }
         uint2 q = __ldcs(Q2 + t);
         q.x &= mmask; q.y &= mmask;
@@ -248,7 +257,10 @@ int cooperative_grid(int *out) {
         BENES_CUDA_TRY(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev));
         if (!coop) return BENES_ERR_CUDA;
         BENES_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-        BENES_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_full_label, kThreads, 0));
+        BENES_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_full_label<false>, kThreads, 0));
+        int per_sm_packed = 0;
+        BENES_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm_packed, k_full_label<true>, kThreads, 0));
+        if (per_sm_packed < per_sm) per_sm = per_sm_packed;
         if (sms < 1 || per_sm < 1) return BENES_ERR_CUDA;
         cached[dev] = sms * per_sm;
     }
@@ -265,12 +277,17 @@ int launch_inverse_clear(uint32_t *fill, size_t total, cudaStream_t s) {
     return BENES_OK;
 }
 
-int launch_inverse_partition_piece(const uint32_t *perm, uint4 *S, void *pairs, uint32_t *fill,
+int launch_inverse_partition_piece(const uint32_t *perm, void *S, bool packed, void *pairs, uint32_t *fill,
                                    size_t total, size_t j_first, size_t count, int log2m,
                                    cudaStream_t s) {
     const uint32_t buckets = uint32_t(total >> kBucketLog2);
-    k_inverse_partition<<<unsigned(count / kPartChunk), kPartThreads, size_t(buckets) * 8, s>>>(
-        perm, S, static_cast<uint2 *>(pairs), fill, buckets, (1u << log2m) - 1u, j_first);
+    const unsigned grid = unsigned(count / kPartChunk);
+    if (packed)
+        k_inverse_partition<true><<<grid, kPartThreads, size_t(buckets) * 8, s>>>(
+            perm, S, static_cast<uint2 *>(pairs), fill, buckets, log2m, j_first);
+    else
+        k_inverse_partition<false><<<grid, kPartThreads, size_t(buckets) * 8, s>>>(
+            perm, S, static_cast<uint2 *>(pairs), fill, buckets, log2m, j_first);
     return launch_status();
 }
 
@@ -280,23 +297,25 @@ int launch_inverse_scatter(const void *pairs, uint32_t *Q, size_t total, int log
     return launch_status();
 }
 
-int launch_inverse_partitioned(const uint32_t *perm, uint4 *S, uint32_t *Q, void *pairs, uint32_t *fill,
-                               size_t total, int log2m, cudaStream_t s) {
+int launch_inverse_partitioned(const uint32_t *perm, void *S, bool packed, uint32_t *Q, void *pairs,
+                               uint32_t *fill, size_t total, int log2m, cudaStream_t s) {
     int rc;
     if ((rc = launch_inverse_clear(fill, total, s))) return rc;
-    if ((rc = launch_inverse_partition_piece(perm, S, pairs, fill, total, 0, total, log2m, s))) return rc;
+    if ((rc = launch_inverse_partition_piece(perm, S, packed, pairs, fill, total, 0, total, log2m, s)))
+        return rc;
     return launch_inverse_scatter(pairs, Q, total, log2m, s);
 }
 
-int launch_inverse(const uint32_t *perm, uint4 *S, uint32_t *Q, size_t total, int log2m,
+int launch_inverse(const uint32_t *perm, void *S, bool packed, uint32_t *Q, size_t total, int log2m,
                    cudaStream_t s) {
     size_t quads = total / 4;
-    k_inverse<<<grid_for(quads), kThreads, 0, s>>>(reinterpret_cast<const uint4 *>(perm), S, Q,
-                                                   quads, (1u << log2m) - 1u);
+    const uint4 *P4 = reinterpret_cast<const uint4 *>(perm);
+    if (packed) k_inverse<true><<<grid_for(quads), kThreads, 0, s>>>(P4, S, Q, quads, log2m);
+    else k_inverse<false><<<grid_for(quads), kThreads, 0, s>>>(P4, S, Q, quads, log2m);
     return launch_status();
 }
 
-int launch_full_label(const uint4 *S, const uint32_t *Q, unsigned long long *Wd, size_t total,
+int launch_full_label(const void *S, bool packed, const uint32_t *Q, unsigned long long *Wd, size_t total,
                       int log2m, BitsLayout L, int out_stage, const uint32_t *gate,
                       cudaStream_t s) {
     int grid = 0;
@@ -304,25 +323,32 @@ int launch_full_label(const uint4 *S, const uint32_t *Q, unsigned long long *Wd,
     if (rc) return rc;
     size_t need = (total / 2 + kThreads - 1) / kThreads;
     if (size_t(grid) > need) grid = int(need);
-    uint32_t mmask = (1u << log2m) - 1u;
     int passes = log2m - 2;
-    void *args[] = {(void *)&S, (void *)&Q, (void *)&Wd, (void *)&total, (void *)&mmask,
+    void *args[] = {(void *)&S, (void *)&Q, (void *)&Wd, (void *)&total, (void *)&log2m,
                     (void *)&passes, (void *)&L, (void *)&out_stage, (void *)&gate};
-    if (cudaLaunchCooperativeKernel((const void *)k_full_label, dim3(grid), dim3(kThreads), args, 0,
-                                    s) != cudaSuccess) {
+    const void *kernel = packed ? (const void *)k_full_label<true> : (const void *)k_full_label<false>;
+    if (cudaLaunchCooperativeKernel(kernel, dim3(grid), dim3(kThreads), args, 0, s) != cudaSuccess) {
         cudaGetLastError();
         return BENES_ERR_CUDA;
     }
     return launch_status();
 }
 
-int launch_split(const uint4 *S, const uint32_t *Q, uint4 *Sn, uint32_t *Qn, size_t total,
-                 int log2m, BitsLayout L, int in_stage, int out_stage, const uint32_t *gate,
+int launch_split(const void *S, bool packed, const uint32_t *Q, void *Sn, bool next_packed, uint32_t *Qn,
+                 size_t total, int log2m, BitsLayout L, int in_stage, int out_stage, const uint32_t *gate,
                  cudaStream_t s) {
     size_t switches = total / 2;
-    k_split<<<grid_for(switches), kThreads, 0, s>>>(S, reinterpret_cast<const uint2 *>(Q), Sn, Qn,
-                                                    switches, (1u << log2m) - 1u, L, in_stage,
-                                                    out_stage, gate);
+    const uint2 *Q2 = reinterpret_cast<const uint2 *>(Q);
+    const int grid = grid_for(switches);
+    if (packed)          // a packed level is followed by packed levels only
+        k_split<true, true><<<grid, kThreads, 0, s>>>(S, Q2, Sn, Qn, switches, log2m, L, in_stage,
+                                                       out_stage, gate);
+    else if (next_packed)
+        k_split<false, true><<<grid, kThreads, 0, s>>>(S, Q2, Sn, Qn, switches, log2m, L, in_stage,
+                                                        out_stage, gate);
+    else
+        k_split<false, false><<<grid, kThreads, 0, s>>>(S, Q2, Sn, Qn, switches, log2m, L, in_stage,
+                                                         out_stage, gate);
     return launch_status();
 }
 

@@ -58,22 +58,47 @@ __device__ __forceinline__ bool gate_raised(const uint32_t *gate) {
 
 // Step 2.  rulers = T / k threads, launched in index order so that the blocks
 // being walked at any moment are neighbours in memory.
+//
+// Wide records: the walker loads the record (16 B) and claims its owner word
+// with a compare-and-swap.  Packed records: one 64-bit atomic AND with
+// (my code << 2m | ones) returns the two P values and the previous owner and,
+// if the switch was free (owner all ones), leaves my code there; if it was
+// taken, the AND has mangled the other walker's code, and since nobody but the
+// two of us ever touches this switch, writing the old word back repairs it.
+template <bool PACKED>
 __global__ void __launch_bounds__(kThreads)
-k_walk(uint4 *__restrict__ S, const uint32_t *__restrict__ Q, uint4 *__restrict__ rec,
-       uint32_t rulers, uint32_t mmask, int kappa, uint32_t salt, uint32_t cap,
+k_walk(void *__restrict__ Sv, const uint32_t *__restrict__ Q, uint4 *__restrict__ rec,
+       uint32_t rulers, int m, int kappa, uint32_t salt, uint32_t cap,
        uint32_t *__restrict__ gate) {
     const uint32_t rho = blockIdx.x * kThreads + threadIdx.x;
     if (rho >= rulers) return;
+    const uint32_t mmask = (1u << m) - 1u;
     const uint32_t kmask = (1u << kappa) - 1u;
     const uint32_t group = rho >> 1, side0 = rho & 1u;
     const uint32_t t0 = (group << kappa) | ruler_slot(group, salt, kmask);
     uint32_t j = 2u * t0 + side0;
     const uint32_t base = j & ~mmask;
     uint32_t fwd = j, part = kUnowned, peer = rho ^ 1u, hops = 0;
-    uint4 r = __ldcg(S + t0);
-    // the ruler switch belongs to its even-side walker (nobody else claims it)
-    if (!side0) reinterpret_cast<uint32_t *>(S + t0)[2] = rho << 1;
-    uint32_t p = (side0 ? r.x : r.y) & mmask;                     // P[j^1]
+    uint4 *S16 = static_cast<uint4 *>(Sv);
+    unsigned long long *S8 = static_cast<unsigned long long *>(Sv);
+    // packed owners are local to the block: its first ruler output is base >> kappa
+    const uint32_t rho_base = base >> kappa;
+    const int cshift = 2 * m;
+    const unsigned long long low_ones = PACKED ? ((1ull << cshift) - 1ull) : 0ull;
+    const uint32_t none8 = PACKED ? uint32_t(~0ull >> cshift) : 0u;
+
+    uint32_t p;                                                   // P[j^1]
+    if (PACKED) {
+        unsigned long long w;
+        // the ruler switch belongs to its even-side walker (nobody else claims it)
+        if (!side0) w = atomicAnd(S8 + t0, ((unsigned long long)((rho - rho_base) << 1) << cshift) | low_ones);
+        else w = __ldcg(S8 + t0);
+        p = uint32_t(w >> (side0 ? 0 : m)) & mmask;
+    } else {
+        const uint4 r = __ldcg(S16 + t0);
+        if (!side0) reinterpret_cast<uint32_t *>(S16 + t0)[2] = rho << 1;
+        p = (side0 ? r.x : r.y) & mmask;
+    }
     uint32_t q = __ldcg(Q + base + (p ^ 1u)) & mmask;
     for (;;) {
         j = base + q;
@@ -87,17 +112,31 @@ k_walk(uint4 *__restrict__ S, const uint32_t *__restrict__ Q, uint4 *__restrict_
             break;
         }
         if ((hops & 63u) == 0u && gate_raised(gate)) break;       // the level is relabelled anyway
-        r = __ldcg(S + t);
-        p = (side ? r.x : r.y) & mmask;
-        // next hop's gather, issued before the claim is known (harmless if we stop)
-        const uint32_t qn = __ldcg(Q + base + (p ^ 1u)) & mmask;
-        uint32_t prev = r.z;
-        if (prev == kUnowned)
-            prev = atomicCAS(reinterpret_cast<uint32_t *>(S + t) + 2, kUnowned, (rho << 1) | side);
-        if (prev != kUnowned) {                                   // met the walker from the other end
-            peer = prev >> 1;
-            break;
+        uint32_t qn;
+        bool met;
+        if (PACKED) {
+            const unsigned long long mine = (unsigned long long)(((rho - rho_base) << 1) | side) << cshift;
+            const unsigned long long w = atomicAnd(S8 + t, mine | low_ones);
+            p = uint32_t(w >> (side ? 0 : m)) & mmask;
+            // next hop's gather, issued before the claim is looked at (harmless if we stop)
+            qn = __ldcg(Q + base + (p ^ 1u)) & mmask;
+            const uint32_t prev = uint32_t(w >> cshift);
+            met = prev != none8;
+            if (met) {
+                __stcg(S8 + t, w);                                // put the other walker's code back
+                peer = rho_base + (prev >> 1);
+            }
+        } else {
+            const uint4 r = __ldcg(S16 + t);
+            p = (side ? r.x : r.y) & mmask;
+            qn = __ldcg(Q + base + (p ^ 1u)) & mmask;
+            uint32_t prev = r.z;
+            if (prev == kUnowned)
+                prev = atomicCAS(reinterpret_cast<uint32_t *>(S16 + t) + 2, kUnowned, (rho << 1) | side);
+            met = prev != kUnowned;
+            if (met) peer = prev >> 1;
         }
+        if (met) break;                                           // met the walker from the other end
         fwd = min(fwd, j);
         part = min(part, j ^ 1u);
         q = qn;
@@ -252,29 +291,46 @@ k_list_bits(const unsigned long long *__restrict__ W, uint32_t *__restrict__ cb,
 // level; they exchange them with a shuffle and store whole records (owner
 // reset).  If the gate is raised afterwards, the split kernel redoes the
 // records from the relabelled stage.
+template <bool PACKED, bool NEXT_PACKED>
 __global__ void __launch_bounds__(kThreads)
-k_colour(const uint4 *__restrict__ S, const uint32_t *__restrict__ Q,
-         const uint32_t *__restrict__ cb, uint4 *__restrict__ Sn, size_t switches,
-         uint32_t rulers, uint32_t mmask, BitsLayout L, int out_stage, uint32_t cap,
+k_colour(const void *__restrict__ S, const uint32_t *__restrict__ Q,
+         const uint32_t *__restrict__ cb, void *__restrict__ Sn, size_t switches,
+         uint32_t rulers, int m, int kappa, BitsLayout L, int out_stage, uint32_t cap,
          uint32_t *__restrict__ gate) {
     const size_t stride = size_t(gridDim.x) * blockDim.x;
+    const uint32_t mmask = (1u << m) - 1u;
     const uint32_t H = (mmask + 1) >> 1;
     for (size_t t = size_t(blockIdx.x) * blockDim.x + threadIdx.x; t < switches; t += stride) {
-        const uint4 r = __ldcs(S + t);
-        const uint32_t code = r.z;
+        const size_t base = (2 * t) & ~size_t(mmask);
+        uint32_t px, py, code;
+        bool owned;
+        if (PACKED) {
+            const unsigned long long w = __ldcs(static_cast<const unsigned long long *>(S) + t);
+            px = uint32_t(w) & mmask;
+            py = uint32_t(w >> m) & mmask;
+            const uint32_t local = uint32_t(w >> (2 * m));
+            owned = local != uint32_t(~0ull >> (2 * m));
+            code = (uint32_t(base >> kappa) << 1) + local;      // owner local to the block -> global
+        } else {
+            const uint4 r = __ldcs(static_cast<const uint4 *>(S) + t);
+            px = r.x & mmask;
+            py = r.y & mmask;
+            code = r.z;
+            owned = code != kUnowned;
+        }
         uint32_t c;
-        if (code != kUnowned) {
+        if (owned) {
             const uint32_t rho = code >> 1;
             const uint32_t rr = rho < rulers ? rho : 0u;
             c = ((__ldg(cb + (rr >> 5)) >> (rr & 31u)) ^ code) & 1u;
         } else {
             // loop without ruler: walk the g-cycle of output 2t
             const uint32_t j0 = uint32_t(2 * t);
-            const uint32_t base = j0 & ~mmask;
+            const uint32_t b32 = uint32_t(base);
             uint32_t j = j0, mn = j0, hops = 0;
             for (;;) {
-                const uint32_t p = rec_p(S, j ^ 1u) & mmask;
-                j = base + (__ldg(Q + base + (p ^ 1u)) & mmask);
+                const uint32_t p = rec_p<PACKED>(S, j ^ 1u, m);
+                j = b32 + (__ldg(Q + b32 + (p ^ 1u)) & mmask);
                 if (j == j0) break;
                 if (++hops > cap) {
                     *gate = 1u;
@@ -287,15 +343,13 @@ k_colour(const uint4 *__restrict__ S, const uint32_t *__restrict__ Q,
         }
         const uint32_t word = __ballot_sync(0xFFFFFFFFu, c);
         if ((threadIdx.x & 31) == 0) L.bits[L.word(out_stage, t >> 5)] = word;
-        const size_t base = (2 * t) & ~size_t(mmask);
         const uint32_t tl = uint32_t(t - base / 2);
-        const uint32_t px = r.x & mmask, py = r.y & mmask;
         const uint32_t up = (c ? py : px) >> 1, lo = (c ? px : py) >> 1;
         const uint32_t got = __shfl_xor_sync(0xFFFFFFFFu, (tl & 1u) ? up : lo, 1);
         if (tl & 1u)
-            Sn[(base >> 1) + (H >> 1) + (tl >> 1)] = make_uint4(got, lo, kUnowned, 0u);
+            rec_write<NEXT_PACKED>(Sn, (base >> 1) + (H >> 1) + (tl >> 1), m - 1, got, lo);
         else
-            Sn[(base >> 1) + (tl >> 1)] = make_uint4(up, got, kUnowned, 0u);
+            rec_write<NEXT_PACKED>(Sn, (base >> 1) + (tl >> 1), m - 1, up, got);
     }
 }
 
@@ -350,15 +404,15 @@ int sampled_scratch_reset(const SampledScratch &sc, size_t total, int kappa, cud
     return BENES_OK;
 }
 
-int sampled_label(uint4 *S, const uint32_t *Q, uint4 *Sn, const SampledScratch &sc, size_t total,
-                  int log2m, int kappa, uint32_t salt, uint32_t cap, BitsLayout L, int out_stage,
-                  uint32_t *gate, cudaStream_t s) {
-    const uint32_t mmask = (1u << log2m) - 1u;
+int sampled_label(void *S, bool packed, const uint32_t *Q, void *Sn, bool next_packed,
+                  const SampledScratch &sc, size_t total, int log2m, int kappa, uint32_t salt,
+                  uint32_t cap, BitsLayout L, int out_stage, uint32_t *gate, cudaStream_t s) {
     const uint32_t R = uint32_t(total >> kappa);
     const unsigned rgrid = (R + kThreads - 1) / kThreads;
     {
         ProfileScope ps(kWalk, s);
-        k_walk<<<rgrid, kThreads, 0, s>>>(S, Q, sc.rec, R, mmask, kappa, salt, cap, gate);
+        if (packed) k_walk<true><<<rgrid, kThreads, 0, s>>>(S, Q, sc.rec, R, log2m, kappa, salt, cap, gate);
+        else k_walk<false><<<rgrid, kThreads, 0, s>>>(S, Q, sc.rec, R, log2m, kappa, salt, cap, gate);
         int rc = launch_status();
         if (rc) return rc;
     }
@@ -410,8 +464,16 @@ int sampled_label(uint4 *S, const uint32_t *Q, uint4 *Sn, const SampledScratch &
         const size_t switches = total / 2;
         size_t blocks = (switches + kThreads - 1) / kThreads;
         const size_t capb = size_t(kSMs) * 8;
-        k_colour<<<unsigned(blocks < capb ? blocks : capb), kThreads, 0, s>>>(
-            S, Q, cb, Sn, switches, R, mmask, L, out_stage, cap, gate);
+        const unsigned grid = unsigned(blocks < capb ? blocks : capb);
+        if (packed)          // a packed level is followed by packed levels only
+            k_colour<true, true><<<grid, kThreads, 0, s>>>(S, Q, cb, Sn, switches, R, log2m, kappa, L,
+                                                            out_stage, cap, gate);
+        else if (next_packed)
+            k_colour<false, true><<<grid, kThreads, 0, s>>>(S, Q, cb, Sn, switches, R, log2m, kappa, L,
+                                                             out_stage, cap, gate);
+        else
+            k_colour<false, false><<<grid, kThreads, 0, s>>>(S, Q, cb, Sn, switches, R, log2m, kappa, L,
+                                                              out_stage, cap, gate);
         return launch_status();
     }
 }
