@@ -75,7 +75,7 @@ def algorithmic_bytes_per_element(kind: str, ebytes: int, kappa: int) -> float:
 NCU_DRAM_BYTES_PER_ELEMENT = {
     # mean over the 10 k_walk launches of one route at N = 2^25 (profiles/k_walk_n2p25.md),
     # scaled by the elements of a launch; the top level of a larger N moves somewhat more
-    "walk": 38.3,
+    "walk": 32.8,
 }
 FALLBACK_HBM_GBS = 6650.0
 RANDOM_GATHER_PEAK_G = 64.7
