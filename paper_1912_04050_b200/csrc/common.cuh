@@ -110,6 +110,28 @@ __device__ __forceinline__ uint32_t rec_p(const void *S, uint32_t j, int m) {
     return static_cast<const uint32_t *>(S)[(size_t(j >> 1) << 2) | (j & 1u)] & ((1u << m) - 1u);
 }
 
+// bits a (16) and b (16) interleaved: bit 2i = a_i, bit 2i+1 = b_i
+__device__ __forceinline__ uint32_t interleave16(uint32_t a, uint32_t b) {
+    uint32_t x = (a & 0xFFFFu) | (b << 16);
+    // outer perfect shuffle of the two halves
+    uint32_t t;
+    t = (x ^ (x >> 8)) & 0x0000FF00u; x ^= t ^ (t << 8);
+    t = (x ^ (x >> 4)) & 0x00F000F0u; x ^= t ^ (t << 4);
+    t = (x ^ (x >> 2)) & 0x0C0C0C0Cu; x ^= t ^ (t << 2);
+    t = (x ^ (x >> 1)) & 0x22222222u; x ^= t ^ (t << 1);
+    return x;
+}
+
+// A thread of the streaming kernels owns the two neighbouring switches 2i and
+// 2i+1; a warp therefore covers 64 switches = two stage words.  c0 / c1 = the
+// bit of the thread's first / second switch.
+__device__ __forceinline__ void store_stage_bits64(uint32_t *row_words, uint32_t c0, uint32_t c1) {
+    const uint32_t b0 = __ballot_sync(0xFFFFFFFFu, c0), b1 = __ballot_sync(0xFFFFFFFFu, c1);
+    const uint32_t lane = threadIdx.x & 31u;
+    if (lane == 0) row_words[0] = interleave16(b0, b1);
+    if (lane == 1) row_words[1] = interleave16(b0 >> 16, b1 >> 16);
+}
+
 // an unowned record of a level with blocks of 2^m outputs
 template <bool PACKED>
 __device__ __forceinline__ void rec_write(void *S, size_t t, int m, uint32_t p0, uint32_t p1) {

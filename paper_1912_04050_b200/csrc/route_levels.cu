@@ -197,37 +197,42 @@ k_full_label(const void *__restrict__ S, const uint32_t *__restrict__ Q,
 // level; they exchange them with a shuffle and store whole records.
 template <bool PACKED, bool NEXT_PACKED>
 __global__ void __launch_bounds__(kThreads)
-k_split(const void *__restrict__ S, const uint2 *__restrict__ Q2, void *__restrict__ Sn,
-        uint32_t *__restrict__ Qn, size_t switches, int m, BitsLayout L, int in_stage,
+k_split(const void *__restrict__ S, const uint4 *__restrict__ Q4, void *__restrict__ Sn,
+        uint32_t *__restrict__ Qn, uint32_t pairs, int m, BitsLayout L, int in_stage,
         int out_stage, const uint32_t *__restrict__ gate) {
     const bool with_records = !gate || *gate != 0u;
     const uint32_t mmask = (1u << m) - 1u;
-    size_t stride = size_t(gridDim.x) * blockDim.x;
+    const uint32_t stride = gridDim.x * blockDim.x;
     const uint32_t H = (mmask + 1) >> 1;
-    for (size_t t = size_t(blockIdx.x) * blockDim.x + threadIdx.x; t < switches; t += stride) {
-        size_t base = (2 * t) & ~size_t(mmask);
-        uint32_t tl = uint32_t(t - base / 2);
+    // a thread owns the neighbouring switches t = 2i and t + 1 (inputs 2t .. 2t+3)
+    for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < pairs; i += stride) {
+        const uint32_t t = 2u * i;
+        const uint32_t base = (2u * t) & ~mmask;
+        const uint32_t tl = t - (base >> 1);
+        const size_t row = L.word(out_stage, (base >> 1) >> 5);      // the block's words of that stage
+        const uint32_t *colours = L.bits + row;
         if (with_records) {
-            uint32_t px, py;
-            rec_read<PACKED>(S, t, m, px, py);
-            // colour of output 2t
-            uint32_t c = (L.bits[L.word(out_stage, t >> 5)] >> (t & 31)) & 1u;
-            uint32_t up = (c ? py : px) >> 1, lo = (c ? px : py) >> 1;
-            uint32_t got = __shfl_xor_sync(0xFFFFFFFFu, (tl & 1u) ? up : lo, 1);
-            if (tl & 1u)
-                rec_write<NEXT_PACKED>(Sn, (base >> 1) + (H >> 1) + (tl >> 1), m - 1, got, lo);
-            else
-                rec_write<NEXT_PACKED>(Sn, (base >> 1) + (tl >> 1), m - 1, up, got);
+            uint32_t px0, py0, px1, py1;
+            rec_read<PACKED>(S, t, m, px0, py0);
+            rec_read<PACKED>(S, t + 1, m, px1, py1);
+            // colours of outputs 2t and 2t+2
+            const uint32_t cwd = colours[tl >> 5];
+            const uint32_t c0 = (cwd >> (tl & 31u)) & 1u, c1 = (cwd >> ((tl + 1u) & 31u)) & 1u;
+            const uint32_t r = (base >> 1) + (tl >> 1);
+            rec_write<NEXT_PACKED>(Sn, r, m - 1, (c0 ? py0 : px0) >> 1, (c1 ? py1 : px1) >> 1);
+            rec_write<NEXT_PACKED>(Sn, r + (H >> 1), m - 1, (c0 ? px0 : py0) >> 1, (c1 ? px1 : py1) >> 1);
         }
-        uint2 q = __ldcs(Q2 + t);
-        q.x &= mmask; q.y &= mmask;
-        // colour of the output fed by input 2t
-        size_t o = base + q.x;
-        uint32_t cin = ((L.bits[L.word(out_stage, o >> 6)] >> ((o >> 1) & 31)) & 1u) ^ (q.x & 1u);
-        uint32_t word = __ballot_sync(0xFFFFFFFFu, cin);
-        if ((threadIdx.x & 31) == 0) L.bits[L.word(in_stage, t >> 5)] = word;
-        Qn[base + cin * H + tl] = q.x >> 1;
-        Qn[base + (1u - cin) * H + tl] = q.y >> 1;
+        uint4 q = __ldcs(Q4 + i);
+        q.x &= mmask; q.y &= mmask; q.z &= mmask; q.w &= mmask;
+        // colour of the output fed by input 2t (2t+2): that output's switch bit, flipped for an odd output
+        const uint32_t cin0 = ((colours[q.x >> 6] >> ((q.x >> 1) & 31u)) ^ q.x) & 1u;
+        const uint32_t cin1 = ((colours[q.z >> 6] >> ((q.z >> 1) & 31u)) ^ q.z) & 1u;
+        store_stage_bits64(L.bits + L.word(in_stage, (t - 2u * (threadIdx.x & 31u)) >> 5), cin0, cin1);
+        // positions tl, tl+1 of the two half-blocks
+        *reinterpret_cast<uint2 *>(Qn + base + tl) =
+            make_uint2((cin0 ? q.y : q.x) >> 1, (cin1 ? q.w : q.z) >> 1);
+        *reinterpret_cast<uint2 *>(Qn + base + H + tl) =
+            make_uint2((cin0 ? q.x : q.y) >> 1, (cin1 ? q.z : q.w) >> 1);
     }
 }
 
@@ -337,17 +342,17 @@ int launch_full_label(const void *S, bool packed, const uint32_t *Q, unsigned lo
 int launch_split(const void *S, bool packed, const uint32_t *Q, void *Sn, bool next_packed, uint32_t *Qn,
                  size_t total, int log2m, BitsLayout L, int in_stage, int out_stage, const uint32_t *gate,
                  cudaStream_t s) {
-    size_t switches = total / 2;
-    const uint2 *Q2 = reinterpret_cast<const uint2 *>(Q);
-    const int grid = grid_for(switches);
+    const uint32_t pairs = uint32_t(total / 4);                  // two switches per thread
+    const uint4 *Q4 = reinterpret_cast<const uint4 *>(Q);
+    const int grid = grid_for(pairs);
     if (packed)          // a packed level is followed by packed levels only
-        k_split<true, true><<<grid, kThreads, 0, s>>>(S, Q2, Sn, Qn, switches, log2m, L, in_stage,
+        k_split<true, true><<<grid, kThreads, 0, s>>>(S, Q4, Sn, Qn, pairs, log2m, L, in_stage,
                                                        out_stage, gate);
     else if (next_packed)
-        k_split<false, true><<<grid, kThreads, 0, s>>>(S, Q2, Sn, Qn, switches, log2m, L, in_stage,
+        k_split<false, true><<<grid, kThreads, 0, s>>>(S, Q4, Sn, Qn, pairs, log2m, L, in_stage,
                                                         out_stage, gate);
     else
-        k_split<false, false><<<grid, kThreads, 0, s>>>(S, Q2, Sn, Qn, switches, log2m, L, in_stage,
+        k_split<false, false><<<grid, kThreads, 0, s>>>(S, Q4, Sn, Qn, pairs, log2m, L, in_stage,
                                                          out_stage, gate);
     return launch_status();
 }

@@ -291,65 +291,72 @@ k_list_bits(const unsigned long long *__restrict__ W, uint32_t *__restrict__ cb,
 // level; they exchange them with a shuffle and store whole records (owner
 // reset).  If the gate is raised afterwards, the split kernel redoes the
 // records from the relabelled stage.
+// colour of output 2t from the owner of switch t, or by walking the cycle
+template <bool PACKED>
+__device__ __forceinline__ uint32_t colour_of(const void *S, const uint32_t *Q, const uint32_t *cb,
+                                              uint32_t t, uint32_t base, bool owned, uint32_t code,
+                                              uint32_t rulers, int m, uint32_t mmask, uint32_t cap,
+                                              uint32_t *gate) {
+    if (owned) {
+        const uint32_t rho = code >> 1;
+        const uint32_t rr = rho < rulers ? rho : 0u;
+        return ((__ldg(cb + (rr >> 5)) >> (rr & 31u)) ^ code) & 1u;
+    }
+    // loop without ruler: walk the g-cycle of output 2t
+    const uint32_t j0 = 2u * t;
+    uint32_t j = j0, mn = j0, hops = 0;
+    for (;;) {
+        const uint32_t p = rec_p<PACKED>(S, j ^ 1u, m);
+        j = base + (__ldg(Q + base + (p ^ 1u)) & mmask);
+        if (j == j0) break;
+        if (++hops > cap) {
+            *gate = 1u;
+            break;
+        }
+        if ((hops & 63u) == 0u && gate_raised(gate)) break;
+        mn = min(mn, j);
+    }
+    return mn & 1u;
+}
+
+// A thread owns the neighbouring switches 2i and 2i+1: their colour-0 outputs
+// are neighbours in the upper half-block of the next level and their colour-1
+// outputs in the lower one, i.e. the thread writes one whole record of each.
 template <bool PACKED, bool NEXT_PACKED>
 __global__ void __launch_bounds__(kThreads)
 k_colour(const void *__restrict__ S, const uint32_t *__restrict__ Q,
-         const uint32_t *__restrict__ cb, void *__restrict__ Sn, size_t switches,
+         const uint32_t *__restrict__ cb, void *__restrict__ Sn, uint32_t pairs,
          uint32_t rulers, int m, int kappa, BitsLayout L, int out_stage, uint32_t cap,
          uint32_t *__restrict__ gate) {
-    const size_t stride = size_t(gridDim.x) * blockDim.x;
+    const uint32_t stride = gridDim.x * blockDim.x;
     const uint32_t mmask = (1u << m) - 1u;
     const uint32_t H = (mmask + 1) >> 1;
-    for (size_t t = size_t(blockIdx.x) * blockDim.x + threadIdx.x; t < switches; t += stride) {
-        const size_t base = (2 * t) & ~size_t(mmask);
-        uint32_t px, py, code;
-        bool owned;
+    for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < pairs; i += stride) {
+        const uint32_t t = 2u * i;                              // first switch of the pair
+        const uint32_t base = (2u * t) & ~mmask;
+        uint32_t px0, py0, px1, py1, code0, code1;
+        bool own0, own1;
         if (PACKED) {
-            const unsigned long long w = __ldcs(static_cast<const unsigned long long *>(S) + t);
-            px = uint32_t(w) & mmask;
-            py = uint32_t(w >> m) & mmask;
-            const uint32_t local = uint32_t(w >> (2 * m));
-            owned = local != uint32_t(~0ull >> (2 * m));
-            code = (uint32_t(base >> kappa) << 1) + local;      // owner local to the block -> global
+            const ulonglong2 w = __ldcs(static_cast<const ulonglong2 *>(S) + i);
+            const uint32_t none = uint32_t(~0ull >> (2 * m)), rb = (base >> kappa) << 1;
+            px0 = uint32_t(w.x) & mmask; py0 = uint32_t(w.x >> m) & mmask;
+            px1 = uint32_t(w.y) & mmask; py1 = uint32_t(w.y >> m) & mmask;
+            const uint32_t l0 = uint32_t(w.x >> (2 * m)), l1 = uint32_t(w.y >> (2 * m));
+            own0 = l0 != none; own1 = l1 != none;
+            code0 = rb + l0; code1 = rb + l1;                    // owner local to the block -> global
         } else {
-            const uint4 r = __ldcs(static_cast<const uint4 *>(S) + t);
-            px = r.x & mmask;
-            py = r.y & mmask;
-            code = r.z;
-            owned = code != kUnowned;
+            const uint4 r0 = __ldcs(static_cast<const uint4 *>(S) + t);
+            const uint4 r1 = __ldcs(static_cast<const uint4 *>(S) + t + 1);
+            px0 = r0.x & mmask; py0 = r0.y & mmask; code0 = r0.z; own0 = code0 != kUnowned;
+            px1 = r1.x & mmask; py1 = r1.y & mmask; code1 = r1.z; own1 = code1 != kUnowned;
         }
-        uint32_t c;
-        if (owned) {
-            const uint32_t rho = code >> 1;
-            const uint32_t rr = rho < rulers ? rho : 0u;
-            c = ((__ldg(cb + (rr >> 5)) >> (rr & 31u)) ^ code) & 1u;
-        } else {
-            // loop without ruler: walk the g-cycle of output 2t
-            const uint32_t j0 = uint32_t(2 * t);
-            const uint32_t b32 = uint32_t(base);
-            uint32_t j = j0, mn = j0, hops = 0;
-            for (;;) {
-                const uint32_t p = rec_p<PACKED>(S, j ^ 1u, m);
-                j = b32 + (__ldg(Q + b32 + (p ^ 1u)) & mmask);
-                if (j == j0) break;
-                if (++hops > cap) {
-                    *gate = 1u;
-                    break;
-                }
-                if ((hops & 63u) == 0u && gate_raised(gate)) break;
-                mn = min(mn, j);
-            }
-            c = mn & 1u;
-        }
-        const uint32_t word = __ballot_sync(0xFFFFFFFFu, c);
-        if ((threadIdx.x & 31) == 0) L.bits[L.word(out_stage, t >> 5)] = word;
-        const uint32_t tl = uint32_t(t - base / 2);
-        const uint32_t up = (c ? py : px) >> 1, lo = (c ? px : py) >> 1;
-        const uint32_t got = __shfl_xor_sync(0xFFFFFFFFu, (tl & 1u) ? up : lo, 1);
-        if (tl & 1u)
-            rec_write<NEXT_PACKED>(Sn, (base >> 1) + (H >> 1) + (tl >> 1), m - 1, got, lo);
-        else
-            rec_write<NEXT_PACKED>(Sn, (base >> 1) + (tl >> 1), m - 1, up, got);
+        const uint32_t c0 = colour_of<PACKED>(S, Q, cb, t, base, own0, code0, rulers, m, mmask, cap, gate);
+        const uint32_t c1 = colour_of<PACKED>(S, Q, cb, t + 1, base, own1, code1, rulers, m, mmask, cap, gate);
+        // a warp covers 64 switches: two words of the output-side stage
+        store_stage_bits64(L.bits + L.word(out_stage, (t - 2u * (threadIdx.x & 31u)) >> 5), c0, c1);
+        const uint32_t r = (base >> 1) + (((t - (base >> 1)) >> 1));   // record of the upper half
+        rec_write<NEXT_PACKED>(Sn, r, m - 1, (c0 ? py0 : px0) >> 1, (c1 ? py1 : px1) >> 1);
+        rec_write<NEXT_PACKED>(Sn, r + (H >> 1), m - 1, (c0 ? px0 : py0) >> 1, (c1 ? px1 : py1) >> 1);
     }
 }
 
@@ -461,8 +468,8 @@ int sampled_label(void *S, bool packed, const uint32_t *Q, void *Sn, bool next_p
         k_list_bits<<<rgrid, kThreads, 0, s>>>(sc.list[0], cb, R);
         int rc = launch_status();
         if (rc) return rc;
-        const size_t switches = total / 2;
-        size_t blocks = (switches + kThreads - 1) / kThreads;
+        const uint32_t switches = uint32_t(total / 4);           // pairs of switches, one per thread
+        size_t blocks = (size_t(switches) + kThreads - 1) / kThreads;
         const size_t capb = size_t(kSMs) * 8;
         const unsigned grid = unsigned(blocks < capb ? blocks : capb);
         if (packed)          // a packed level is followed by packed levels only
