@@ -62,6 +62,13 @@ struct BitsLayout {
         size_t lw = flat_word & ((size_t(1) << log2w) - 1);
         return ((perm * size_t(2 * log2n - 1) + size_t(stage)) << log2w) + lw;
     }
+    // the same in 32 bits: a chunk has at most 2^30 elements, i.e. fewer than
+    // 2^24 * (2n-1) < 2^30 words
+    __host__ __device__ uint32_t word32(int stage, uint32_t flat_word) const {
+        const uint32_t perm = flat_word >> log2w;
+        const uint32_t lw = flat_word & ((1u << log2w) - 1u);
+        return ((perm * uint32_t(2 * log2n - 1) + uint32_t(stage)) << log2w) + lw;
+    }
 };
 
 // ---- layout of a level in HBM ------------------------------------------------
@@ -110,26 +117,19 @@ __device__ __forceinline__ uint32_t rec_p(const void *S, uint32_t j, int m) {
     return static_cast<const uint32_t *>(S)[(size_t(j >> 1) << 2) | (j & 1u)] & ((1u << m) - 1u);
 }
 
-// bits a (16) and b (16) interleaved: bit 2i = a_i, bit 2i+1 = b_i
-__device__ __forceinline__ uint32_t interleave16(uint32_t a, uint32_t b) {
-    uint32_t x = (a & 0xFFFFu) | (b << 16);
-    // outer perfect shuffle of the two halves
-    uint32_t t;
-    t = (x ^ (x >> 8)) & 0x0000FF00u; x ^= t ^ (t << 8);
-    t = (x ^ (x >> 4)) & 0x00F000F0u; x ^= t ^ (t << 4);
-    t = (x ^ (x >> 2)) & 0x0C0C0C0Cu; x ^= t ^ (t << 2);
-    t = (x ^ (x >> 1)) & 0x22222222u; x ^= t ^ (t << 1);
-    return x;
-}
-
 // A thread of the streaming kernels owns the two neighbouring switches 2i and
 // 2i+1; a warp therefore covers 64 switches = two stage words.  c0 / c1 = the
-// bit of the thread's first / second switch.
+// bit of the thread's first / second switch.  Lane l fetches the bits of
+// switches l and 32 + l (held by threads l/2 and 16 + l/2), so that two
+// ballots give the two words.
 __device__ __forceinline__ void store_stage_bits64(uint32_t *row_words, uint32_t c0, uint32_t c1) {
-    const uint32_t b0 = __ballot_sync(0xFFFFFFFFu, c0), b1 = __ballot_sync(0xFFFFFFFFu, c1);
     const uint32_t lane = threadIdx.x & 31u;
-    if (lane == 0) row_words[0] = interleave16(b0, b1);
-    if (lane == 1) row_words[1] = interleave16(b0 >> 16, b1 >> 16);
+    const uint32_t both = c0 | (c1 << 1);
+    const uint32_t lo = __shfl_sync(0xFFFFFFFFu, both, int(lane >> 1));
+    const uint32_t hi = __shfl_sync(0xFFFFFFFFu, both, int(16u + (lane >> 1)));
+    const uint32_t w0 = __ballot_sync(0xFFFFFFFFu, (lo >> (lane & 1u)) & 1u);
+    const uint32_t w1 = __ballot_sync(0xFFFFFFFFu, (hi >> (lane & 1u)) & 1u);
+    if (lane < 2) row_words[lane] = lane ? w1 : w0;
 }
 
 // an unowned record of a level with blocks of 2^m outputs
@@ -144,6 +144,13 @@ __device__ __forceinline__ void rec_write(void *S, size_t t, int m, uint32_t p0,
 
 __device__ __forceinline__ unsigned long long make_word(uint32_t nxt, uint32_t mn) {
     return (static_cast<unsigned long long>(mn) << 32) | nxt;
+}
+
+// The streaming kernels of a level give every CTA `rounds` consecutive groups of
+// `threads` items: as many as keep 8 CTAs per SM of a 148-SM part busy, at most 16.
+inline uint32_t stream_rounds(size_t items, int threads) {
+    const size_t r = items / (size_t(threads) * 148 * 8);
+    return uint32_t(r < 1 ? 1 : (r > 16 ? 16 : r));
 }
 
 // ---- per-level HBM path (route_levels.cu) ----------------------------------

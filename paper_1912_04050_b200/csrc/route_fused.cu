@@ -186,7 +186,7 @@ k_route_fused(const uint32_t *__restrict__ P, int records, uint32_t *__restrict_
         uint16_t *peer = (size_t(M) + size_t(R) * 10 <= size_t(2 * M))
                              ? reinterpret_cast<uint16_t *>(list + R)      // still inside that buffer
                              : reinterpret_cast<uint16_t *>(tail);
-        const bool sampled = logS >= kFMinLogS;
+        const bool sampled = LOGM >= kFMinLogS && logS >= kFMinLogS;
 
         // a1: block-local inverse; owners reset
         for (int j = tid; j < M; j += T) {
@@ -231,7 +231,7 @@ k_route_fused(const uint32_t *__restrict__ P, int records, uint32_t *__restrict_
                     q = qn;
                 }
                 recm[rho] = fwd | (part << 16);
-                peer[rho] = uint16_t(pr < uint32_t(R) ? pr : uint32_t(rho));
+                peer[rho] = uint16_t(pr < uint32_t(R > 0 ? R : 1) ? pr : uint32_t(rho));
             }
             __syncthreads();
             // contracted list: next = peer ^ 1, minimum = own side of mine, far side of the peer's

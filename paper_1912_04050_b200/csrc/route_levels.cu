@@ -196,21 +196,31 @@ k_full_label(const void *__restrict__ S, const uint32_t *__restrict__ Q,
 // so two neighbouring threads hold the two values of one record of the next
 // level; they exchange them with a shuffle and store whole records.
 template <bool PACKED, bool NEXT_PACKED>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 8)
 k_split(const void *__restrict__ S, const uint4 *__restrict__ Q4, void *__restrict__ Sn,
         uint32_t *__restrict__ Qn, uint32_t pairs, int m, BitsLayout L, int in_stage,
-        int out_stage, const uint32_t *__restrict__ gate) {
+        int out_stage, const uint32_t *__restrict__ gate, uint32_t rounds) {
     const bool with_records = !gate || *gate != 0u;
     const uint32_t mmask = (1u << m) - 1u;
-    const uint32_t stride = gridDim.x * blockDim.x;
+    // a CTA takes `rounds` consecutive groups of blockDim.x pairs: the colour
+    // words it gathers belong to one block of the level for a long time (L1 hits)
+    const uint32_t stride = blockDim.x;
+    const uint32_t last = min(pairs, (blockIdx.x + 1u) * rounds * stride);
     const uint32_t H = (mmask + 1) >> 1;
-    // a thread owns the neighbouring switches t = 2i and t + 1 (inputs 2t .. 2t+3)
-    for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < pairs; i += stride) {
+    // a thread owns the neighbouring switches t = 2i and t + 1 (inputs 2t .. 2t+3);
+    // the inverses of the next round are on their way while this one is split
+    // (pairs is a multiple of 32: a warp stays together)
+    uint32_t i = blockIdx.x * rounds * stride + threadIdx.x;
+    uint4 q = make_uint4(0, 0, 0, 0);
+    if (i < last) q = __ldcs(Q4 + i);
+    while (i < last) {
+        const uint32_t inext = i + stride;
+        uint4 qn = make_uint4(0, 0, 0, 0);
+        if (inext < last) qn = __ldcs(Q4 + inext);
         const uint32_t t = 2u * i;
         const uint32_t base = (2u * t) & ~mmask;
         const uint32_t tl = t - (base >> 1);
-        const size_t row = L.word(out_stage, (base >> 1) >> 5);      // the block's words of that stage
-        const uint32_t *colours = L.bits + row;
+        const uint32_t *colours = L.bits + L.word32(out_stage, (base >> 1) >> 5);   // the block's words of that stage
         if (with_records) {
             uint32_t px0, py0, px1, py1;
             rec_read<PACKED>(S, t, m, px0, py0);
@@ -222,17 +232,18 @@ k_split(const void *__restrict__ S, const uint4 *__restrict__ Q4, void *__restri
             rec_write<NEXT_PACKED>(Sn, r, m - 1, (c0 ? py0 : px0) >> 1, (c1 ? py1 : px1) >> 1);
             rec_write<NEXT_PACKED>(Sn, r + (H >> 1), m - 1, (c0 ? px0 : py0) >> 1, (c1 ? px1 : py1) >> 1);
         }
-        uint4 q = __ldcs(Q4 + i);
         q.x &= mmask; q.y &= mmask; q.z &= mmask; q.w &= mmask;
         // colour of the output fed by input 2t (2t+2): that output's switch bit, flipped for an odd output
         const uint32_t cin0 = ((colours[q.x >> 6] >> ((q.x >> 1) & 31u)) ^ q.x) & 1u;
         const uint32_t cin1 = ((colours[q.z >> 6] >> ((q.z >> 1) & 31u)) ^ q.z) & 1u;
-        store_stage_bits64(L.bits + L.word(in_stage, (t - 2u * (threadIdx.x & 31u)) >> 5), cin0, cin1);
+        store_stage_bits64(L.bits + L.word32(in_stage, (t - 2u * (threadIdx.x & 31u)) >> 5), cin0, cin1);
         // positions tl, tl+1 of the two half-blocks
         *reinterpret_cast<uint2 *>(Qn + base + tl) =
             make_uint2((cin0 ? q.y : q.x) >> 1, (cin1 ? q.w : q.z) >> 1);
         *reinterpret_cast<uint2 *>(Qn + base + H + tl) =
             make_uint2((cin0 ? q.x : q.y) >> 1, (cin1 ? q.z : q.w) >> 1);
+        q = qn;
+        i = inext;
     }
 }
 
@@ -344,16 +355,17 @@ int launch_split(const void *S, bool packed, const uint32_t *Q, void *Sn, bool n
                  cudaStream_t s) {
     const uint32_t pairs = uint32_t(total / 4);                  // two switches per thread
     const uint4 *Q4 = reinterpret_cast<const uint4 *>(Q);
-    const int grid = grid_for(pairs);
+    const uint32_t rounds = stream_rounds(pairs, kThreads);
+    const unsigned grid = unsigned((size_t(pairs) + size_t(kThreads) * rounds - 1) / (size_t(kThreads) * rounds));
     if (packed)          // a packed level is followed by packed levels only
         k_split<true, true><<<grid, kThreads, 0, s>>>(S, Q4, Sn, Qn, pairs, log2m, L, in_stage,
-                                                       out_stage, gate);
+                                                       out_stage, gate, rounds);
     else if (next_packed)
         k_split<false, true><<<grid, kThreads, 0, s>>>(S, Q4, Sn, Qn, pairs, log2m, L, in_stage,
-                                                        out_stage, gate);
+                                                        out_stage, gate, rounds);
     else
         k_split<false, false><<<grid, kThreads, 0, s>>>(S, Q4, Sn, Qn, pairs, log2m, L, in_stage,
-                                                         out_stage, gate);
+                                                         out_stage, gate, rounds);
     return launch_status();
 }
 

@@ -41,7 +41,7 @@ namespace benes {
 namespace {
 
 constexpr int kThreads = 256;
-constexpr int kSMs = 148;
+constexpr int kWalkThreads = 128;             // a CTA's slots are free again when its longest walk ends
 constexpr int kListThreads = 1024;
 
 __device__ __forceinline__ uint32_t ruler_slot(uint32_t group, uint32_t salt, uint32_t kmask) {
@@ -66,11 +66,11 @@ __device__ __forceinline__ bool gate_raised(const uint32_t *gate) {
 // taken, the AND has mangled the other walker's code, and since nobody but the
 // two of us ever touches this switch, writing the old word back repairs it.
 template <bool PACKED>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kWalkThreads)
 k_walk(void *__restrict__ Sv, const uint32_t *__restrict__ Q, uint4 *__restrict__ rec,
        uint32_t rulers, int m, int kappa, uint32_t salt, uint32_t cap,
        uint32_t *__restrict__ gate) {
-    const uint32_t rho = blockIdx.x * kThreads + threadIdx.x;
+    const uint32_t rho = blockIdx.x * kWalkThreads + threadIdx.x;
     if (rho >= rulers) return;
     const uint32_t mmask = (1u << m) - 1u;
     const uint32_t kmask = (1u << kappa) - 1u;
@@ -327,36 +327,55 @@ __global__ void __launch_bounds__(kThreads)
 k_colour(const void *__restrict__ S, const uint32_t *__restrict__ Q,
          const uint32_t *__restrict__ cb, void *__restrict__ Sn, uint32_t pairs,
          uint32_t rulers, int m, int kappa, BitsLayout L, int out_stage, uint32_t cap,
-         uint32_t *__restrict__ gate) {
-    const uint32_t stride = gridDim.x * blockDim.x;
+         uint32_t *__restrict__ gate, uint32_t rounds) {
+    // a CTA takes `rounds` consecutive groups of blockDim.x pairs: the ruler bits
+    // it gathers belong to one block of the level for a long time (L1 hits)
+    const uint32_t stride = blockDim.x;
+    const uint32_t last = min(pairs, (blockIdx.x + 1u) * rounds * stride);
     const uint32_t mmask = (1u << m) - 1u;
     const uint32_t H = (mmask + 1) >> 1;
-    for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < pairs; i += stride) {
+    const uint32_t none = PACKED ? uint32_t(~0ull >> (2 * m)) : kUnowned;
+    // the records of the next round are on their way while this one is coloured
+    // (pairs is a multiple of 32: a warp stays together)
+    uint32_t i = blockIdx.x * rounds * stride + threadIdx.x;
+    ulonglong2 w = make_ulonglong2(0, 0);
+    uint4 r0 = make_uint4(0, 0, 0, 0), r1 = r0;
+    if (i < last) {
+        if (PACKED) w = __ldcs(static_cast<const ulonglong2 *>(S) + i);
+        else { r0 = __ldcs(static_cast<const uint4 *>(S) + 2 * size_t(i)); r1 = __ldcs(static_cast<const uint4 *>(S) + 2 * size_t(i) + 1); }
+    }
+    while (i < last) {
+        const uint32_t inext = i + stride;
+        ulonglong2 wn = make_ulonglong2(0, 0);
+        uint4 r0n = make_uint4(0, 0, 0, 0), r1n = r0n;
+        if (inext < last) {
+            if (PACKED) wn = __ldcs(static_cast<const ulonglong2 *>(S) + inext);
+            else { r0n = __ldcs(static_cast<const uint4 *>(S) + 2 * size_t(inext)); r1n = __ldcs(static_cast<const uint4 *>(S) + 2 * size_t(inext) + 1); }
+        }
         const uint32_t t = 2u * i;                              // first switch of the pair
         const uint32_t base = (2u * t) & ~mmask;
         uint32_t px0, py0, px1, py1, code0, code1;
         bool own0, own1;
         if (PACKED) {
-            const ulonglong2 w = __ldcs(static_cast<const ulonglong2 *>(S) + i);
-            const uint32_t none = uint32_t(~0ull >> (2 * m)), rb = (base >> kappa) << 1;
+            const uint32_t rb = (base >> kappa) << 1;
             px0 = uint32_t(w.x) & mmask; py0 = uint32_t(w.x >> m) & mmask;
             px1 = uint32_t(w.y) & mmask; py1 = uint32_t(w.y >> m) & mmask;
             const uint32_t l0 = uint32_t(w.x >> (2 * m)), l1 = uint32_t(w.y >> (2 * m));
             own0 = l0 != none; own1 = l1 != none;
             code0 = rb + l0; code1 = rb + l1;                    // owner local to the block -> global
         } else {
-            const uint4 r0 = __ldcs(static_cast<const uint4 *>(S) + t);
-            const uint4 r1 = __ldcs(static_cast<const uint4 *>(S) + t + 1);
-            px0 = r0.x & mmask; py0 = r0.y & mmask; code0 = r0.z; own0 = code0 != kUnowned;
-            px1 = r1.x & mmask; py1 = r1.y & mmask; code1 = r1.z; own1 = code1 != kUnowned;
+            px0 = r0.x & mmask; py0 = r0.y & mmask; code0 = r0.z; own0 = code0 != none;
+            px1 = r1.x & mmask; py1 = r1.y & mmask; code1 = r1.z; own1 = code1 != none;
         }
         const uint32_t c0 = colour_of<PACKED>(S, Q, cb, t, base, own0, code0, rulers, m, mmask, cap, gate);
         const uint32_t c1 = colour_of<PACKED>(S, Q, cb, t + 1, base, own1, code1, rulers, m, mmask, cap, gate);
         // a warp covers 64 switches: two words of the output-side stage
-        store_stage_bits64(L.bits + L.word(out_stage, (t - 2u * (threadIdx.x & 31u)) >> 5), c0, c1);
+        store_stage_bits64(L.bits + L.word32(out_stage, (t - 2u * (threadIdx.x & 31u)) >> 5), c0, c1);
         const uint32_t r = (base >> 1) + (((t - (base >> 1)) >> 1));   // record of the upper half
         rec_write<NEXT_PACKED>(Sn, r, m - 1, (c0 ? py0 : px0) >> 1, (c1 ? py1 : px1) >> 1);
         rec_write<NEXT_PACKED>(Sn, r + (H >> 1), m - 1, (c0 ? px0 : py0) >> 1, (c1 ? px1 : py1) >> 1);
+        w = wn; r0 = r0n; r1 = r1n;
+        i = inext;
     }
 }
 
@@ -418,8 +437,9 @@ int sampled_label(void *S, bool packed, const uint32_t *Q, void *Sn, bool next_p
     const unsigned rgrid = (R + kThreads - 1) / kThreads;
     {
         ProfileScope ps(kWalk, s);
-        if (packed) k_walk<true><<<rgrid, kThreads, 0, s>>>(S, Q, sc.rec, R, log2m, kappa, salt, cap, gate);
-        else k_walk<false><<<rgrid, kThreads, 0, s>>>(S, Q, sc.rec, R, log2m, kappa, salt, cap, gate);
+        const unsigned wgrid = (R + kWalkThreads - 1) / kWalkThreads;
+        if (packed) k_walk<true><<<wgrid, kWalkThreads, 0, s>>>(S, Q, sc.rec, R, log2m, kappa, salt, cap, gate);
+        else k_walk<false><<<wgrid, kWalkThreads, 0, s>>>(S, Q, sc.rec, R, log2m, kappa, salt, cap, gate);
         int rc = launch_status();
         if (rc) return rc;
     }
@@ -469,18 +489,17 @@ int sampled_label(void *S, bool packed, const uint32_t *Q, void *Sn, bool next_p
         int rc = launch_status();
         if (rc) return rc;
         const uint32_t switches = uint32_t(total / 4);           // pairs of switches, one per thread
-        size_t blocks = (size_t(switches) + kThreads - 1) / kThreads;
-        const size_t capb = size_t(kSMs) * 8;
-        const unsigned grid = unsigned(blocks < capb ? blocks : capb);
+        const uint32_t rounds = stream_rounds(switches, kThreads);
+        const unsigned grid = unsigned((size_t(switches) + size_t(kThreads) * rounds - 1) / (size_t(kThreads) * rounds));
         if (packed)          // a packed level is followed by packed levels only
             k_colour<true, true><<<grid, kThreads, 0, s>>>(S, Q, cb, Sn, switches, R, log2m, kappa, L,
-                                                            out_stage, cap, gate);
+                                                            out_stage, cap, gate, rounds);
         else if (next_packed)
             k_colour<false, true><<<grid, kThreads, 0, s>>>(S, Q, cb, Sn, switches, R, log2m, kappa, L,
-                                                             out_stage, cap, gate);
+                                                             out_stage, cap, gate, rounds);
         else
             k_colour<false, false><<<grid, kThreads, 0, s>>>(S, Q, cb, Sn, switches, R, log2m, kappa, L,
-                                                              out_stage, cap, gate);
+                                                              out_stage, cap, gate, rounds);
         return launch_status();
     }
 }
