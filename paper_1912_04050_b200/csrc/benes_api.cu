@@ -146,7 +146,7 @@ int route_levels(const uint32_t *perm, int n, size_t batch, uint32_t *bits, char
     {
         ProfileScope ps(kInverse, s);
         // the 64-bit word array is free until the first level is labelled
-        // (the bucketed form needs whole buckets of 2^18 entries)
+        // (the bucketed form needs whole buckets, of 2^18 entries at most)
         const bool bucketed = g_inverse_partitioned && T >= (size_t(1) << kInversePartitionMinLog2) &&
                               (T & ((size_t(1) << 18) - 1)) == 0;
         const int pieces = hp ? hp->pieces : 0;

@@ -60,27 +60,44 @@ k_inverse(const uint4 *__restrict__ P4, void *__restrict__ S, uint32_t *__restri
 }
 
 // a1 for large inputs, as two streaming passes instead of one pass of random
-// 4-byte writes.  Q is cut into buckets of 2^kBucketLog2 consecutive entries (a
-// piece that stays in L2).  Pass 1 reads P in order, writes the switch records
-// and appends (destination, source) pairs to the bucket of the destination: a
-// CTA counts its 8192 elements per bucket in shared memory, reserves room in
-// every bucket with one global atomic per bucket, then writes its pairs there.
-// A bucket of a permutation receives exactly as many pairs as it has entries;
-// for other inputs positions wrap inside the bucket, so every access stays in
-// bounds.  Pass 2 reads the pairs bucket by bucket and scatters inside the
-// bucket's piece of Q.
-constexpr int kBucketLog2 = 18;
+// 4-byte writes.  Q is cut into buckets of 2^blog consecutive entries.  Pass 1
+// reads P in order, writes the switch records and appends (destination,
+// source) pairs to the bucket of the destination: a CTA counts its 8192
+// elements per bucket in shared memory (the count an element sees is its rank
+// among the CTA's elements of that bucket), reserves room in every bucket with
+// one global atomic per bucket, sorts its pairs by bucket in shared memory and
+// writes them out in that order, so that the pairs of one bucket leave as one
+// run of consecutive 8-byte entries (whole sectors instead of 32 scattered
+// stores per warp).  A bucket of a permutation receives exactly as many pairs
+// as it has entries; for other inputs positions wrap inside the bucket, so
+// every access stays in bounds.  Pass 2 reads the pairs bucket by bucket and
+// scatters inside the bucket's piece of Q: with buckets of 2^15 entries a CTA
+// builds the piece in shared memory and writes it out in order; with buckets
+// of 2^18 entries (inputs of more than 2^27 elements, whose 2^15-entry
+// buckets would be too many for the counters) the piece stays in L2.
+constexpr int kBucketSmemLog2 = 15;
+constexpr int kBucketL2Log2 = 18;
 constexpr int kPartChunk = 8192;
 constexpr int kPartThreads = 1024;
+
+inline int bucket_log2(size_t total) {
+    return (total >> kBucketSmemLog2) <= size_t(kInverseMaxBuckets) ? kBucketSmemLog2 : kBucketL2Log2;
+}
+inline size_t partition_smem(uint32_t buckets) { return size_t(kPartChunk) * 8 + size_t(buckets) * 12; }
 
 template <bool PACKED>
 __global__ void __launch_bounds__(kPartThreads)
 k_inverse_partition(const uint32_t *__restrict__ P, void *__restrict__ S, uint2 *__restrict__ pairs,
-                    uint32_t *__restrict__ fill, uint32_t buckets, int m, size_t j_first) {
+                    uint32_t *__restrict__ fill, uint32_t buckets, int blog, int m, size_t j_first) {
     const uint32_t mmask = (1u << m) - 1u;
-    extern __shared__ uint32_t sh[];           // count[buckets], then offset[buckets]
-    uint32_t *count = sh, *offset = sh + buckets;
-    for (uint32_t b = threadIdx.x; b < buckets; b += kPartThreads) count[b] = 0u;
+    extern __shared__ __align__(8) unsigned char part_smem[];
+    uint2 *stage = reinterpret_cast<uint2 *>(part_smem);                  // the CTA's pairs, sorted by bucket
+    uint32_t *count = reinterpret_cast<uint32_t *>(stage + kPartChunk);  // per bucket: elements of this CTA
+    uint32_t *first = count + buckets;                                    // ... where they start in `stage`
+    uint32_t *offset = first + buckets;                                   // ... and in the bucket
+    __shared__ uint32_t warp_sum[kPartThreads / 32];
+    const uint32_t tid = threadIdx.x, lane = tid & 31u, wid = tid >> 5;
+    for (uint32_t b = tid; b < buckets; b += kPartThreads) count[b] = 0u;
     __syncthreads();
     const size_t j0 = j_first + size_t(blockIdx.x) * kPartChunk;
     constexpr int kPer = kPartChunk / kPartThreads;
@@ -88,37 +105,93 @@ k_inverse_partition(const uint32_t *__restrict__ P, void *__restrict__ S, uint2 
 #pragma unroll
     for (int i = 0; i < kPer; i += 2) {
         // two values = one switch
-        const size_t j = j0 + 2 * (size_t(i / 2) * kPartThreads + threadIdx.x);
+        const size_t j = j0 + 2 * (size_t(i / 2) * kPartThreads + tid);
         const uint2 p = __ldcs(reinterpret_cast<const uint2 *>(P + j));
         const uint32_t px = p.x & mmask, py = p.y & mmask;
         rec_write<PACKED>(S, j >> 1, m, px, py);
         const uint32_t base = uint32_t(j) & ~mmask;
         dest[i] = base + px;
         dest[i + 1] = base + py;
-        rank[i] = atomicAdd(count + (dest[i] >> kBucketLog2), 1u);
-        rank[i + 1] = atomicAdd(count + (dest[i + 1] >> kBucketLog2), 1u);
+        rank[i] = atomicAdd(count + (dest[i] >> blog), 1u);
+        rank[i + 1] = atomicAdd(count + (dest[i + 1] >> blog), 1u);
     }
     __syncthreads();
-    for (uint32_t b = threadIdx.x; b < buckets; b += kPartThreads)
-        offset[b] = count[b] ? atomicAdd(fill + b, count[b]) : 0u;
+    // exclusive prefix sum of the counts: a thread takes `per` consecutive buckets
+    const uint32_t per = (buckets + kPartThreads - 1) / kPartThreads;
+    const uint32_t b_lo = min(tid * per, buckets), b_hi = min(b_lo + per, buckets);
+    uint32_t mine = 0;
+    for (uint32_t b = b_lo; b < b_hi; ++b) mine += count[b];
+    uint32_t incl = mine;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+        if (lane >= uint32_t(d)) incl += v;
+    }
+    if (lane == 31) warp_sum[wid] = incl;
     __syncthreads();
-    constexpr uint32_t kInBucket = (1u << kBucketLog2) - 1u;
+    if (wid == 0) {
+        const uint32_t w = warp_sum[lane];
+        uint32_t wi = w;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, wi, d);
+            if (lane >= uint32_t(d)) wi += v;
+        }
+        warp_sum[lane] = wi - w;
+    }
+    __syncthreads();
+    uint32_t run = warp_sum[wid] + incl - mine;
+    for (uint32_t b = b_lo; b < b_hi; ++b) {
+        const uint32_t c = count[b];
+        first[b] = run;
+        run += c;
+        offset[b] = c ? atomicAdd(fill + b, c) : 0u;
+    }
+    __syncthreads();
 #pragma unroll
     for (int i = 0; i < kPer; ++i) {
-        const size_t j = j0 + 2 * (size_t(i / 2) * kPartThreads + threadIdx.x) + (i & 1);
-        const uint32_t b = dest[i] >> kBucketLog2;
-        const uint32_t slot = (offset[b] + rank[i]) & kInBucket;
-        pairs[(size_t(b) << kBucketLog2) + slot] = make_uint2(dest[i], uint32_t(j) & mmask);
+        const size_t j = j0 + 2 * (size_t(i / 2) * kPartThreads + tid) + (i & 1);
+        stage[first[dest[i] >> blog] + rank[i]] = make_uint2(dest[i], uint32_t(j) & mmask);
+    }
+    __syncthreads();
+    const uint32_t in_bucket = (1u << blog) - 1u;
+    for (uint32_t k = tid; k < uint32_t(kPartChunk); k += kPartThreads) {
+        const uint2 pr = stage[k];
+        const uint32_t b = pr.x >> blog;
+        const uint32_t slot = (offset[b] + (k - first[b])) & in_bucket;
+        pairs[(size_t(b) << blog) + slot] = pr;
     }
 }
 
+// Pass 2, buckets of 2^kBucketSmemLog2 entries: one CTA per bucket.
+__global__ void __launch_bounds__(1024)
+k_inverse_scatter_smem(const uint2 *__restrict__ pairs, uint32_t *__restrict__ Q, uint32_t mmask) {
+    extern __shared__ __align__(16) uint32_t piece[];
+    constexpr uint32_t kEntries = 1u << kBucketSmemLog2, kInBucket = kEntries - 1u;
+    const size_t b0 = size_t(blockIdx.x) << kBucketSmemLog2;
+    // entries no pair names (only possible if the input is not a permutation) read as 0
+    for (uint32_t k = threadIdx.x; k < kEntries / 4; k += 1024)
+        reinterpret_cast<uint4 *>(piece)[k] = make_uint4(0, 0, 0, 0);
+    __syncthreads();
+    const uint4 *src = reinterpret_cast<const uint4 *>(pairs + b0);      // two pairs per load
+    for (uint32_t k = threadIdx.x; k < kEntries / 2; k += 1024) {
+        const uint4 two = __ldcs(src + k);
+        piece[two.x & kInBucket] = two.y & mmask;
+        piece[two.z & kInBucket] = two.w & mmask;
+    }
+    __syncthreads();
+    uint4 *dst = reinterpret_cast<uint4 *>(Q + b0);
+    for (uint32_t k = threadIdx.x; k < kEntries / 4; k += 1024) dst[k] = reinterpret_cast<const uint4 *>(piece)[k];
+}
+
+// Pass 2, buckets of 2^kBucketL2Log2 entries.
 __global__ void __launch_bounds__(kThreads)
 k_inverse_scatter(const uint2 *__restrict__ pairs, uint32_t *__restrict__ Q, size_t total, uint32_t mmask) {
     const size_t i = size_t(blockIdx.x) * kThreads + threadIdx.x;
     if (i >= total) return;
     const uint2 pr = __ldcs(pairs + i);
     // the destination is forced into the bucket this pair sits in
-    constexpr uint32_t kInBucket = (1u << kBucketLog2) - 1u;
+    constexpr uint32_t kInBucket = (1u << kBucketL2Log2) - 1u;
     const size_t d = (i & ~size_t(kInBucket)) | (pr.x & kInBucket);
     Q[d] = pr.y & mmask;
 }
@@ -289,27 +362,42 @@ int cooperative_grid(int *out) {
 // Pass 1 over elements [j_first, j_first + count) (a multiple of 8192); `fill`
 // must have been cleared before the first piece.  Pass 2 over everything.
 int launch_inverse_clear(uint32_t *fill, size_t total, cudaStream_t s) {
-    BENES_CUDA_TRY(cudaMemsetAsync(fill, 0, (total >> kBucketLog2) * 4, s));
+    BENES_CUDA_TRY(cudaMemsetAsync(fill, 0, (total >> bucket_log2(total)) * 4, s));
     return BENES_OK;
 }
 
 int launch_inverse_partition_piece(const uint32_t *perm, void *S, bool packed, void *pairs, uint32_t *fill,
                                    size_t total, size_t j_first, size_t count, int log2m,
                                    cudaStream_t s) {
-    const uint32_t buckets = uint32_t(total >> kBucketLog2);
+    const int blog = bucket_log2(total);
+    const uint32_t buckets = uint32_t(total >> blog);
     const unsigned grid = unsigned(count / kPartChunk);
+    const size_t smem = partition_smem(buckets);
+    static bool configured = false;
+    if (!configured) {
+        const int most = int(partition_smem(kInverseMaxBuckets));
+        BENES_CUDA_TRY(cudaFuncSetAttribute(k_inverse_partition<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most));
+        BENES_CUDA_TRY(cudaFuncSetAttribute(k_inverse_partition<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, most));
+        BENES_CUDA_TRY(cudaFuncSetAttribute(k_inverse_scatter_smem, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            4 << kBucketSmemLog2));
+        configured = true;
+    }
     if (packed)
-        k_inverse_partition<true><<<grid, kPartThreads, size_t(buckets) * 8, s>>>(
-            perm, S, static_cast<uint2 *>(pairs), fill, buckets, log2m, j_first);
+        k_inverse_partition<true><<<grid, kPartThreads, smem, s>>>(
+            perm, S, static_cast<uint2 *>(pairs), fill, buckets, blog, log2m, j_first);
     else
-        k_inverse_partition<false><<<grid, kPartThreads, size_t(buckets) * 8, s>>>(
-            perm, S, static_cast<uint2 *>(pairs), fill, buckets, log2m, j_first);
+        k_inverse_partition<false><<<grid, kPartThreads, smem, s>>>(
+            perm, S, static_cast<uint2 *>(pairs), fill, buckets, blog, log2m, j_first);
     return launch_status();
 }
 
 int launch_inverse_scatter(const void *pairs, uint32_t *Q, size_t total, int log2m, cudaStream_t s) {
-    k_inverse_scatter<<<unsigned((total + kThreads - 1) / kThreads), kThreads, 0, s>>>(
-        static_cast<const uint2 *>(pairs), Q, total, (1u << log2m) - 1u);
+    if (bucket_log2(total) == kBucketSmemLog2)
+        k_inverse_scatter_smem<<<unsigned(total >> kBucketSmemLog2), 1024, 4 << kBucketSmemLog2, s>>>(
+            static_cast<const uint2 *>(pairs), Q, (1u << log2m) - 1u);
+    else
+        k_inverse_scatter<<<unsigned((total + kThreads - 1) / kThreads), kThreads, 0, s>>>(
+            static_cast<const uint2 *>(pairs), Q, total, (1u << log2m) - 1u);
     return launch_status();
 }
 
