@@ -86,7 +86,7 @@ inline int bucket_log2(size_t total) {
 inline size_t partition_smem(uint32_t buckets) { return size_t(kPartChunk) * 8 + size_t(buckets) * 12; }
 
 template <bool PACKED>
-__global__ void __launch_bounds__(kPartThreads)
+__global__ void __launch_bounds__(kPartThreads, 2)
 k_inverse_partition(const uint32_t *__restrict__ P, void *__restrict__ S, uint2 *__restrict__ pairs,
                     uint32_t *__restrict__ fill, uint32_t buckets, int blog, int m, size_t j_first) {
     const uint32_t mmask = (1u << m) - 1u;
@@ -174,10 +174,14 @@ k_inverse_scatter_smem(const uint2 *__restrict__ pairs, uint32_t *__restrict__ Q
         reinterpret_cast<uint4 *>(piece)[k] = make_uint4(0, 0, 0, 0);
     __syncthreads();
     const uint4 *src = reinterpret_cast<const uint4 *>(pairs + b0);      // two pairs per load
-    for (uint32_t k = threadIdx.x; k < kEntries / 2; k += 1024) {
-        const uint4 two = __ldcs(src + k);
-        piece[two.x & kInBucket] = two.y & mmask;
-        piece[two.z & kInBucket] = two.w & mmask;
+    constexpr int kLoads = int(kEntries / 2 / 1024);                     // all of a thread's loads in flight
+    uint4 two[kLoads];
+#pragma unroll
+    for (int i = 0; i < kLoads; ++i) two[i] = __ldcs(src + threadIdx.x + i * 1024);
+#pragma unroll
+    for (int i = 0; i < kLoads; ++i) {
+        piece[two[i].x & kInBucket] = two[i].y & mmask;
+        piece[two[i].z & kInBucket] = two[i].w & mmask;
     }
     __syncthreads();
     uint4 *dst = reinterpret_cast<uint4 *>(Q + b0);
