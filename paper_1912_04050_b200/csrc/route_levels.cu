@@ -447,7 +447,12 @@ int launch_split(const void *S, bool packed, const uint32_t *Q, void *Sn, bool n
                  cudaStream_t s) {
     const uint32_t pairs = uint32_t(total / 4);                  // two switches per thread
     const uint4 *Q4 = reinterpret_cast<const uint4 *>(Q);
-    const uint32_t rounds = stream_rounds(pairs, kThreads);
+    // Colour words are gathered at random from the block's row of the output-side
+    // stage (2^(m-1) bits).  Rows of 32 KiB and less stay in L1 whatever the CTAs
+    // of an SM work on; for rows of 64 to 256 KiB the CTAs that are resident
+    // together (8 per SM) should cover about one block, so that an SM sees one row.
+    uint32_t rounds = stream_rounds(pairs, kThreads);
+    if (log2m >= 20 && log2m <= 22 && rounds > (1u << (log2m - 20))) rounds = 1u << (log2m - 20);
     const unsigned grid = unsigned((size_t(pairs) + size_t(kThreads) * rounds - 1) / (size_t(kThreads) * rounds));
     if (packed)          // a packed level is followed by packed levels only
         k_split<true, true><<<grid, kThreads, 0, s>>>(S, Q4, Sn, Qn, pairs, log2m, L, in_stage,
