@@ -335,6 +335,11 @@ k_colour(const void *__restrict__ S, const uint32_t *__restrict__ Q,
     const uint32_t mmask = (1u << m) - 1u;
     const uint32_t H = (mmask + 1) >> 1;
     const uint32_t none = PACKED ? uint32_t(~0ull >> (2 * m)) : kUnowned;
+    // packed fields with 32-bit operations (m < 32): the owner starts at bit 2m of
+    // the word, the next level's owner (all ones) at bit 2(m-1)
+    const int s_own = 2 * m, s_next = 2 * (m - 1);
+    const uint32_t ones_lo = s_next < 32 ? ~0u << s_next : 0u;
+    const uint32_t ones_hi = s_next < 32 ? ~0u : ~0u << (s_next - 32);
     // the records of the next round are on their way while this one is coloured
     // (pairs is a multiple of 32: a warp stays together)
     uint32_t i = blockIdx.x * rounds * stride + threadIdx.x;
@@ -358,22 +363,40 @@ k_colour(const void *__restrict__ S, const uint32_t *__restrict__ Q,
         bool own0, own1;
         if (PACKED) {
             const uint32_t rb = (base >> kappa) << 1;
-            px0 = uint32_t(w.x) & mmask; py0 = uint32_t(w.x >> m) & mmask;
-            px1 = uint32_t(w.y) & mmask; py1 = uint32_t(w.y >> m) & mmask;
-            const uint32_t l0 = uint32_t(w.x >> (2 * m)), l1 = uint32_t(w.y >> (2 * m));
+            const uint32_t lo0 = uint32_t(w.x), hi0 = uint32_t(w.x >> 32);
+            const uint32_t lo1 = uint32_t(w.y), hi1 = uint32_t(w.y >> 32);
+            px0 = lo0 & mmask; py0 = __funnelshift_r(lo0, hi0, m) & mmask;
+            px1 = lo1 & mmask; py1 = __funnelshift_r(lo1, hi1, m) & mmask;
+            const uint32_t l0 = s_own >= 32 ? hi0 >> (s_own - 32) : __funnelshift_r(lo0, hi0, s_own);
+            const uint32_t l1 = s_own >= 32 ? hi1 >> (s_own - 32) : __funnelshift_r(lo1, hi1, s_own);
             own0 = l0 != none; own1 = l1 != none;
             code0 = rb + l0; code1 = rb + l1;                    // owner local to the block -> global
         } else {
             px0 = r0.x & mmask; py0 = r0.y & mmask; code0 = r0.z; own0 = code0 != none;
             px1 = r1.x & mmask; py1 = r1.y & mmask; code1 = r1.z; own1 = code1 != none;
         }
-        const uint32_t c0 = colour_of<PACKED>(S, Q, cb, t, base, own0, code0, rulers, m, mmask, cap, gate);
-        const uint32_t c1 = colour_of<PACKED>(S, Q, cb, t + 1, base, own1, code1, rulers, m, mmask, cap, gate);
+        uint32_t c0, c1;
+        if (own0 && own1) {                                     // all but the switches of loops without ruler
+            const uint32_t a = (code0 >> 1) < rulers ? code0 >> 1 : 0u, b = (code1 >> 1) < rulers ? code1 >> 1 : 0u;
+            c0 = ((__ldg(cb + (a >> 5)) >> (a & 31u)) ^ code0) & 1u;
+            c1 = ((__ldg(cb + (b >> 5)) >> (b & 31u)) ^ code1) & 1u;
+        } else {
+            c0 = colour_of<PACKED>(S, Q, cb, t, base, own0, code0, rulers, m, mmask, cap, gate);
+            c1 = colour_of<PACKED>(S, Q, cb, t + 1, base, own1, code1, rulers, m, mmask, cap, gate);
+        }
         // a warp covers 64 switches: two words of the output-side stage
         store_stage_bits64(L.bits + L.word32(out_stage, (t - 2u * (threadIdx.x & 31u)) >> 5), c0, c1);
         const uint32_t r = (base >> 1) + (((t - (base >> 1)) >> 1));   // record of the upper half
-        rec_write<NEXT_PACKED>(Sn, r, m - 1, (c0 ? py0 : px0) >> 1, (c1 ? py1 : px1) >> 1);
-        rec_write<NEXT_PACKED>(Sn, r + (H >> 1), m - 1, (c0 ? px0 : py0) >> 1, (c1 ? px1 : py1) >> 1);
+        const uint32_t u0 = (c0 ? py0 : px0) >> 1, u1 = (c1 ? py1 : px1) >> 1;     // upper half-block
+        const uint32_t d0 = (c0 ? px0 : py0) >> 1, d1 = (c1 ? px1 : py1) >> 1;     // lower half-block
+        if (NEXT_PACKED) {
+            uint2 *Sn8 = static_cast<uint2 *>(Sn);
+            Sn8[r] = make_uint2(u0 | (u1 << (m - 1)) | ones_lo, (u1 >> (33 - m)) | ones_hi);
+            Sn8[r + (H >> 1)] = make_uint2(d0 | (d1 << (m - 1)) | ones_lo, (d1 >> (33 - m)) | ones_hi);
+        } else {
+            rec_write<false>(Sn, r, m - 1, u0, u1);
+            rec_write<false>(Sn, r + (H >> 1), m - 1, d0, d1);
+        }
         w = wn; r0 = r0n; r1 = r1n;
         i = inext;
     }
