@@ -190,11 +190,15 @@ k_list_walk(const unsigned long long *__restrict__ W, uint32_t *__restrict__ own
 
 // Step 4, back from a sampled list: every word takes the cycle minimum of its
 // owner (and hands the owner slot back as kUnowned); a word without owner
-// walks its own cycle.
+// walks its own cycle.  For the first list (the rulers of the level) only the
+// parity of the minimum is needed afterwards: with `cb` the kernel writes one
+// bit per word there and leaves the words alone, so that the colouring kernel
+// gathers from an array 64 times smaller than the list (it stays in L1/L2 next
+// to the streaming traffic).  count is a multiple of 32.
 __global__ void __launch_bounds__(kThreads)
 k_list_resolve(unsigned long long *__restrict__ W, uint32_t *__restrict__ owner,
                const unsigned long long *__restrict__ W2, uint32_t count, uint32_t wmask,
-               uint32_t cap, uint32_t *__restrict__ gate) {
+               uint32_t cap, uint32_t *__restrict__ gate, uint32_t *__restrict__ cb) {
     const uint32_t e0 = blockIdx.x * kThreads + threadIdx.x;
     if (e0 >= count) return;
     const uint32_t o = owner[e0];
@@ -217,7 +221,12 @@ k_list_resolve(unsigned long long *__restrict__ W, uint32_t *__restrict__ owner,
             e = uint32_t(v) & wmask;
         }
     }
-    __stcg(W + e0, make_word(uint32_t(w), mn));
+    if (cb) {
+        const uint32_t word = __ballot_sync(0xFFFFFFFFu, mn & 1u);
+        if ((threadIdx.x & 31) == 0) cb[e0 >> 5] = word;
+    } else {
+        __stcg(W + e0, make_word(uint32_t(w), mn));
+    }
 }
 
 // Step 4, the end of the recursion: one CTA labels one block's list of
@@ -226,9 +235,11 @@ k_list_resolve(unsigned long long *__restrict__ W, uint32_t *__restrict__ owner,
 // 2^log2b / PER).  A cycle has at most 2^log2b words (a list sampled from a
 // list need not split evenly between a cycle and its mirror image), hence
 // log2b passes.
+// With `cb` (first list of a level) the parities of the minima go there, one bit
+// per word, instead of the words back to W.
 template <int PER>
 __global__ void __launch_bounds__(kListThreads)
-k_list_label(unsigned long long *__restrict__ W, int log2b) {
+k_list_label(unsigned long long *__restrict__ W, int log2b, uint32_t *__restrict__ cb) {
     extern __shared__ unsigned long long sm[];
     const uint32_t B = 1u << log2b, bmask = B - 1u;
     const size_t base = size_t(blockIdx.x) << log2b;
@@ -257,12 +268,17 @@ k_list_label(unsigned long long *__restrict__ W, int log2b) {
     for (int i = 0; i < PER; ++i) {
         const uint32_t e = tid + uint32_t(i) * T;
         const unsigned long long w = sm[e];
-        W[base + e] = make_word(uint32_t(base) + uint32_t(w), uint32_t(w >> 32));
+        if (cb) {
+            const uint32_t word = __ballot_sync(0xFFFFFFFFu, uint32_t(w >> 32) & 1u);
+            if ((tid & 31u) == 0u) cb[(base + e) >> 5] = word;
+        } else {
+            W[base + e] = make_word(uint32_t(base) + uint32_t(w), uint32_t(w >> 32));
+        }
     }
 }
 
 template <int PER>
-int launch_list_label(unsigned long long *W, uint32_t count, int beta, cudaStream_t s) {
+int launch_list_label(unsigned long long *W, uint32_t count, int beta, uint32_t *cb, cudaStream_t s) {
     static bool configured = false;
     const size_t smem = (size_t(1) << beta) * 8;
     if (!configured) {
@@ -270,19 +286,8 @@ int launch_list_label(unsigned long long *W, uint32_t count, int beta, cudaStrea
                                             (1 << kListSmemLog2) * 8));
         configured = true;
     }
-    k_list_label<PER><<<count >> beta, (1u << beta) / PER, smem, s>>>(W, beta);
+    k_list_label<PER><<<count >> beta, (1u << beta) / PER, smem, s>>>(W, beta, cb);
     return launch_status();
-}
-
-// Between steps 4 and 5: parity of every ruler's cycle minimum, one bit each,
-// so that the colouring kernel gathers from an array 64 times smaller than
-// the list (it stays in L1/L2 next to the streaming traffic).
-__global__ void __launch_bounds__(kThreads)
-k_list_bits(const unsigned long long *__restrict__ W, uint32_t *__restrict__ cb, uint32_t rulers) {
-    const uint32_t rho = blockIdx.x * kThreads + threadIdx.x;     // rulers is a multiple of 32
-    const uint32_t bit = rho < rulers ? (uint32_t(__ldcs(W + rho) >> 32) & 1u) : 0u;
-    const uint32_t word = __ballot_sync(0xFFFFFFFFu, bit);
-    if ((threadIdx.x & 31) == 0 && rho < rulers) cb[rho >> 5] = word;
 }
 
 // Step 5 + output side of the level's switches + the next level's records:
@@ -472,6 +477,8 @@ int sampled_label(void *S, bool packed, const uint32_t *Q, void *Sn, bool next_p
         int rc = launch_status();
         if (rc) return rc;
     }
+    // the walk records are dead: their memory takes the rulers' colour bits
+    uint32_t *cb = reinterpret_cast<uint32_t *>(sc.rec);
     // label the contracted list: sample it until a block's list fits one CTA
     int beta = log2m - kappa;
     const int depth = list_depth(beta);
@@ -491,26 +498,22 @@ int sampled_label(void *S, bool packed, const uint32_t *Q, void *Sn, bool next_p
         ProfileScope ps(kListLabel, s);
         if (beta > kListSmemLog2 || beta < 5) return BENES_ERR_BADARG;
         // 4 words per thread up to 2^12 words, then 1024 threads
-        int rc = beta <= 12 ? launch_list_label<4>(sc.list[depth], count, beta, s)
-               : beta == 13 ? launch_list_label<8>(sc.list[depth], count, beta, s)
-                            : launch_list_label<16>(sc.list[depth], count, beta, s);
+        uint32_t *bits_out = depth == 0 ? cb : nullptr;
+        int rc = beta <= 12 ? launch_list_label<4>(sc.list[depth], count, beta, bits_out, s)
+               : beta == 13 ? launch_list_label<8>(sc.list[depth], count, beta, bits_out, s)
+                            : launch_list_label<16>(sc.list[depth], count, beta, bits_out, s);
         if (rc) return rc;
     }
     for (int d = depth - 1; d >= 0; --d) {
         ProfileScope ps(kListResolve, s);
         const uint32_t c = R >> (kListKappa * d);
         k_list_resolve<<<(c + kThreads - 1) / kThreads, kThreads, 0, s>>>(
-            sc.list[d], sc.owner[d], sc.list[d + 1], c, c - 1u, cap, gate);
+            sc.list[d], sc.owner[d], sc.list[d + 1], c, c - 1u, cap, gate, d == 0 ? cb : nullptr);
         int rc = launch_status();
         if (rc) return rc;
     }
-    // the walk records are dead: their memory takes the rulers' colour bits
-    uint32_t *cb = reinterpret_cast<uint32_t *>(sc.rec);
     {
         ProfileScope ps(kColour, s);
-        k_list_bits<<<rgrid, kThreads, 0, s>>>(sc.list[0], cb, R);
-        int rc = launch_status();
-        if (rc) return rc;
         const uint32_t switches = uint32_t(total / 4);           // pairs of switches, one per thread
         const uint32_t rounds = stream_rounds(switches, kThreads);
         const unsigned grid = unsigned((size_t(switches) + size_t(kThreads) * rounds - 1) / (size_t(kThreads) * rounds));
