@@ -35,7 +35,7 @@ namespace {
 constexpr int kChunkLog2 = 13;               // elements per CTA
 constexpr int kChunk = 1 << kChunkLog2;
 constexpr int kRound = 3;                    // stages between barriers
-constexpr int kApplyThreads = 512;           // two 8-slot groups per thread and round, two CTAs per SM
+constexpr int kApplyThreads = 512;           // two 8-slot groups per thread and round
 
 // Slot u lives at shared-memory index phys(u): an XOR swizzle of the low bits,
 // chosen so that every access pattern of the kernels (consecutive slots; the
@@ -191,7 +191,7 @@ k_apply_inner(const uint32_t *__restrict__ bits, const E *__restrict__ x, E *__r
 // chunk; output side (OUT = true): stages 2n-2-(l0+k-1) .. 2n-2-l0, chunk
 // gathered from its 2^k runs and written contiguously.
 template <typename E, bool OUT>
-__global__ void __launch_bounds__(kApplyThreads, 2)
+__global__ void __launch_bounds__(kApplyThreads, 3)
 k_apply_outer(const uint32_t *__restrict__ bits, const E *__restrict__ x, E *__restrict__ y, int n,
               int l0, int k) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -250,6 +250,9 @@ int apply_fused_typed(const uint32_t *bits, const E *in, E *out, E *scratch, int
     const size_t total = batch << n;
     // payload slots + the switch words of up to 2*13-1 stages
     const size_t smem = size_t(kSmemElems) * sizeof(E) + size_t(2 * kChunkLog2 - 1) * kBitWords * 4;
+    // an outer pass stages the words of at most 7 stages: three CTAs of 8-byte
+    // elements fit one SM, so that one CTA's copies overlap the others' stages
+    const size_t smem_outer = size_t(kSmemElems) * sizeof(E) + size_t(7) * kBitWords * 4;
     static bool configured = false;
     if (!configured) {
         int rc;
@@ -274,7 +277,7 @@ int apply_fused_typed(const uint32_t *bits, const E *in, E *out, E *scratch, int
     int l0 = 0;
     for (int i = 0; i < per_side; ++i) {
         E *dst = next_dst();
-        k_apply_outer<E, false><<<chunks, kApplyThreads, smem, s>>>(bits, src, dst, n, l0, ks[i]);
+        k_apply_outer<E, false><<<chunks, kApplyThreads, smem_outer, s>>>(bits, src, dst, n, l0, ks[i]);
         int rc = launch_status();
         if (rc) return rc;
         src = dst;
@@ -293,7 +296,7 @@ int apply_fused_typed(const uint32_t *bits, const E *in, E *out, E *scratch, int
     for (int i = per_side - 1; i >= 0; --i) {
         E *dst = next_dst();
         l0 -= ks[i];
-        k_apply_outer<E, true><<<chunks, kApplyThreads, smem, s>>>(bits, src, dst, n, l0, ks[i]);
+        k_apply_outer<E, true><<<chunks, kApplyThreads, smem_outer, s>>>(bits, src, dst, n, l0, ks[i]);
         int rc = launch_status();
         if (rc) return rc;
         src = dst;

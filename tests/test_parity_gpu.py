@@ -283,12 +283,13 @@ def test_route_batch_in_chunks():
     assert np.array_equal(gpu_route(perm, n), want)
 
 
-def test_route_n2p28_properties():
+@pytest.mark.parametrize("n", [27, 28], ids=["n2p27", "n2p28"])
+def test_route_large_properties(n):
     """Beyond what the oracle finishes in reasonable time: the routed identity
     payload must reproduce the permutation, and under the canonical rule the
     first output switch of every block of every level is straight (output 0 of a
-    block is the smallest output of its loop)."""
-    n = 28
+    block is the smallest output of its loop).  2^27 is the largest input whose
+    level-0 inverse uses buckets of 2^15 entries, 2^28 uses buckets of 2^18."""
     perm = inputs.random_perm(n, 5)
     d_perm = dev(perm)
     bits = torch.empty(binding.benes_switch_words(n, 1), dtype=torch.int32, device="cuda")
