@@ -253,13 +253,12 @@ int apply_fused_typed(const uint32_t *bits, const E *in, E *out, E *scratch, int
     // an outer pass stages the words of at most 7 stages: three CTAs of 8-byte
     // elements fit one SM, so that one CTA's copies overlap the others' stages
     const size_t smem_outer = size_t(kSmemElems) * sizeof(E) + size_t(7) * kBitWords * 4;
-    static bool configured = false;
-    if (!configured) {
+    static OncePerDevice configured;
+    if (configured.first_use()) {
         int rc;
         if ((rc = opt_in_smem(k_apply_inner<E>, smem))) return rc;
         if ((rc = opt_in_smem(k_apply_outer<E, false>, smem))) return rc;
         if ((rc = opt_in_smem(k_apply_outer<E, true>, smem))) return rc;
-        configured = true;
     }
     const int b = n < kChunkLog2 ? n : kChunkLog2;
     const int outer = n - b;                       // levels handled by the outer kernels, per side

@@ -7,7 +7,6 @@
 namespace benes {
 namespace {
 
-constexpr int kMaxDevices = 64;
 constexpr size_t kAlign = 256;
 // Flat elements processed together by the per-level path (indices are 32 bit).
 int g_chunk_log2 = 30;

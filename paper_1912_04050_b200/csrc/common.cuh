@@ -36,6 +36,21 @@ inline int launch_status() {
     return cudaGetLastError() == cudaSuccess ? BENES_OK : BENES_ERR_CUDA;
 }
 
+// Kernel attributes (opt-in shared memory) belong to a device: a launcher sets
+// them the first time it runs on each device of the process.
+constexpr int kMaxDevices = 64;
+struct OncePerDevice {
+    bool done[kMaxDevices] = {};
+    // true if the caller still has to configure the current device
+    bool first_use() {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return true;
+        if (done[dev]) return false;
+        done[dev] = true;
+        return true;
+    }
+};
+
 // Optional event timing of a group of launches of one kind (see benes.h).
 enum ProfileKind {
     kInverse = 0, kFullLabel, kSplit, kFused, kApply, kWalk, kCombine, kListWalk, kListLabel,

@@ -351,15 +351,14 @@ k_route_fused(const uint32_t *__restrict__ P, int records, uint32_t *__restrict_
 template <int LOGM>
 int launch_one(const uint32_t *P, int records, size_t total, uint32_t *bits, int log2n, cudaStream_t s) {
     using C = FusedCfg<LOGM>;
-    static bool configured = false;
-    if (!configured && C::kSmemBytes > 48 * 1024) {
+    static OncePerDevice configured;
+    if (C::kSmemBytes > 48 * 1024 && configured.first_use()) {
         BENES_CUDA_TRY(cudaFuncSetAttribute(k_route_fused<LOGM>,
                                             cudaFuncAttributeMaxDynamicSharedMemorySize,
                                             int(C::kSmemBytes)));
         BENES_CUDA_TRY(cudaFuncSetAttribute(k_route_fused<LOGM>,
                                             cudaFuncAttributePreferredSharedMemoryCarveout,
                                             cudaSharedmemCarveoutMaxShared));
-        configured = true;
     }
     size_t blocks = total >> LOGM;
     k_route_fused<LOGM><<<unsigned(blocks), C::kThreads, C::kSmemBytes, s>>>(P, records, bits, log2n);

@@ -377,14 +377,13 @@ int launch_inverse_partition_piece(const uint32_t *perm, void *S, bool packed, v
     const uint32_t buckets = uint32_t(total >> blog);
     const unsigned grid = unsigned(count / kPartChunk);
     const size_t smem = partition_smem(buckets);
-    static bool configured = false;
-    if (!configured) {
+    static OncePerDevice configured;
+    if (configured.first_use()) {
         const int most = int(partition_smem(kInverseMaxBuckets));
         BENES_CUDA_TRY(cudaFuncSetAttribute(k_inverse_partition<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most));
         BENES_CUDA_TRY(cudaFuncSetAttribute(k_inverse_partition<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, most));
         BENES_CUDA_TRY(cudaFuncSetAttribute(k_inverse_scatter_smem, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                             4 << kBucketSmemLog2));
-        configured = true;
     }
     if (packed)
         k_inverse_partition<true><<<grid, kPartThreads, smem, s>>>(

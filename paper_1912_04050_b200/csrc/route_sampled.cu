@@ -279,12 +279,11 @@ k_list_label(unsigned long long *__restrict__ W, int log2b, uint32_t *__restrict
 
 template <int PER>
 int launch_list_label(unsigned long long *W, uint32_t count, int beta, uint32_t *cb, cudaStream_t s) {
-    static bool configured = false;
+    static OncePerDevice configured;
     const size_t smem = (size_t(1) << beta) * 8;
-    if (!configured) {
+    if (configured.first_use()) {
         BENES_CUDA_TRY(cudaFuncSetAttribute(k_list_label<PER>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                             (1 << kListSmemLog2) * 8));
-        configured = true;
     }
     k_list_label<PER><<<count >> beta, (1u << beta) / PER, smem, s>>>(W, beta, cb);
     return launch_status();
