@@ -299,18 +299,18 @@ int launch_list_label(unsigned long long *W, uint32_t count, int beta, uint32_t 
 template <bool PACKED>
 __device__ __forceinline__ uint32_t colour_of(const void *S, const uint32_t *Q, const uint32_t *cb,
                                               uint32_t t, uint32_t base, bool owned, uint32_t code,
-                                              uint32_t rulers, int m, uint32_t mmask, uint32_t cap,
-                                              uint32_t *gate) {
+                                              uint32_t p_odd, uint32_t rulers, int m, uint32_t mmask,
+                                              uint32_t cap, uint32_t *gate) {
     if (owned) {
         const uint32_t rho = code >> 1;
         const uint32_t rr = rho < rulers ? rho : 0u;
         return ((__ldg(cb + (rr >> 5)) >> (rr & 31u)) ^ code) & 1u;
     }
-    // loop without ruler: walk the g-cycle of output 2t
+    // loop without ruler: walk the g-cycle of output 2t (p_odd = P[2t+1], which
+    // the caller holds already, starts the first hop)
     const uint32_t j0 = 2u * t;
-    uint32_t j = j0, mn = j0, hops = 0;
+    uint32_t j = j0, mn = j0, hops = 0, p = p_odd;
     for (;;) {
-        const uint32_t p = rec_p<PACKED>(S, j ^ 1u, m);
         j = base + (__ldg(Q + base + (p ^ 1u)) & mmask);
         if (j == j0) break;
         if (++hops > cap) {
@@ -319,8 +319,39 @@ __device__ __forceinline__ uint32_t colour_of(const void *S, const uint32_t *Q, 
         }
         if ((hops & 63u) == 0u && gate_raised(gate)) break;
         mn = min(mn, j);
+        p = rec_p<PACKED>(S, j ^ 1u, m);
     }
     return mn & 1u;
+}
+
+// Both switches of a thread on loops without ruler (the rule for inputs such as
+// the identity, a bit reversal or a transpose, whose loops have one or two
+// switches): the two cycles are walked side by side, so that their gathers
+// overlap.  p0 / p1 = P[2t+1] / P[2t+3].
+template <bool PACKED>
+__device__ __forceinline__ void colour_two_walks(const void *S, const uint32_t *Q, uint32_t t, uint32_t base,
+                                                 uint32_t p0, uint32_t p1, int m, uint32_t mmask,
+                                                 uint32_t cap, uint32_t *gate, uint32_t &c0, uint32_t &c1) {
+    const uint32_t ja = 2u * t, jb = ja + 2u;
+    uint32_t j0 = ja, j1 = jb, mn0 = ja, mn1 = jb, hops = 0;
+    bool run0 = true, run1 = true;
+    while (run0 || run1) {
+        uint32_t q0 = 0, q1 = 0;
+        if (run0) q0 = __ldg(Q + base + (p0 ^ 1u));
+        if (run1) q1 = __ldg(Q + base + (p1 ^ 1u));
+        if (run0) { j0 = base + (q0 & mmask); run0 = j0 != ja; }
+        if (run1) { j1 = base + (q1 & mmask); run1 = j1 != jb; }
+        if (!(run0 || run1)) break;
+        if (++hops > cap) {
+            *gate = 1u;
+            break;
+        }
+        if ((hops & 63u) == 0u && gate_raised(gate)) break;
+        if (run0) { mn0 = min(mn0, j0); p0 = rec_p<PACKED>(S, j0 ^ 1u, m); }
+        if (run1) { mn1 = min(mn1, j1); p1 = rec_p<PACKED>(S, j1 ^ 1u, m); }
+    }
+    c0 = mn0 & 1u;
+    c1 = mn1 & 1u;
 }
 
 // A thread owns the neighbouring switches 2i and 2i+1: their colour-0 outputs
@@ -384,9 +415,11 @@ k_colour(const void *__restrict__ S, const uint32_t *__restrict__ Q,
             const uint32_t a = (code0 >> 1) < rulers ? code0 >> 1 : 0u, b = (code1 >> 1) < rulers ? code1 >> 1 : 0u;
             c0 = ((__ldg(cb + (a >> 5)) >> (a & 31u)) ^ code0) & 1u;
             c1 = ((__ldg(cb + (b >> 5)) >> (b & 31u)) ^ code1) & 1u;
+        } else if (!own0 && !own1) {
+            colour_two_walks<PACKED>(S, Q, t, base, py0, py1, m, mmask, cap, gate, c0, c1);
         } else {
-            c0 = colour_of<PACKED>(S, Q, cb, t, base, own0, code0, rulers, m, mmask, cap, gate);
-            c1 = colour_of<PACKED>(S, Q, cb, t + 1, base, own1, code1, rulers, m, mmask, cap, gate);
+            c0 = colour_of<PACKED>(S, Q, cb, t, base, own0, code0, py0, rulers, m, mmask, cap, gate);
+            c1 = colour_of<PACKED>(S, Q, cb, t + 1, base, own1, code1, py1, rulers, m, mmask, cap, gate);
         }
         // a warp covers 64 switches: two words of the output-side stage
         store_stage_bits64(L.bits + L.word32(out_stage, (t - 2u * (threadIdx.x & 31u)) >> 5), c0, c1);
