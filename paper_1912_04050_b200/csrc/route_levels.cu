@@ -270,8 +270,8 @@ k_full_label(const void *__restrict__ S, const uint32_t *__restrict__ Q,
 // in-side half of a5 + a6: input-side stage word and Q'.  With `with_records`
 // (no sampled labelling, or its gate raised) also the next level's records:
 // position tl of the upper half-block takes P[2t or 2t+1] >> 1 of switch tl,
-// so two neighbouring threads hold the two values of one record of the next
-// level; they exchange them with a shuffle and store whole records.
+// so the thread that owns switches 2i and 2i+1 holds both values of one record
+// of each half-block and stores whole records.
 template <bool PACKED, bool NEXT_PACKED>
 __global__ void __launch_bounds__(kThreads, 8)
 k_split(const void *__restrict__ S, const uint4 *__restrict__ Q4, void *__restrict__ Sn,

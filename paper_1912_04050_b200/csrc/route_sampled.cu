@@ -289,13 +289,7 @@ int launch_list_label(unsigned long long *W, uint32_t count, int beta, uint32_t 
     return launch_status();
 }
 
-// Step 5 + output side of the level's switches + the next level's records:
-// position tl of a half-block takes one of the two P values of switch tl, so
-// two neighbouring threads hold the two values of one record of the next
-// level; they exchange them with a shuffle and store whole records (owner
-// reset).  If the gate is raised afterwards, the split kernel redoes the
-// records from the relabelled stage.
-// colour of output 2t from the owner of switch t, or by walking the cycle
+// Step 5: colour of output 2t from the owner of switch t, or by walking the cycle.
 template <bool PACKED>
 __device__ __forceinline__ uint32_t colour_of(const void *S, const uint32_t *Q, const uint32_t *cb,
                                               uint32_t t, uint32_t base, bool owned, uint32_t code,
@@ -354,9 +348,12 @@ __device__ __forceinline__ void colour_two_walks(const void *S, const uint32_t *
     c1 = mn1 & 1u;
 }
 
-// A thread owns the neighbouring switches 2i and 2i+1: their colour-0 outputs
-// are neighbours in the upper half-block of the next level and their colour-1
-// outputs in the lower one, i.e. the thread writes one whole record of each.
+// Step 5 + output side of the level's switches + the next level's records
+// (owner reset).  A thread owns the neighbouring switches 2i and 2i+1: their
+// colour-0 outputs are neighbours in the upper half-block of the next level and
+// their colour-1 outputs in the lower one, i.e. the thread writes one whole
+// record of each.  If the gate is raised afterwards, the split kernel redoes
+// the records from the relabelled stage.
 template <bool PACKED, bool NEXT_PACKED>
 __global__ void __launch_bounds__(kThreads)
 k_colour(const void *__restrict__ S, const uint32_t *__restrict__ Q,
