@@ -167,8 +167,12 @@ int route_levels(const uint32_t *perm, int n, size_t batch, uint32_t *bits, char
         }
         if (rc) return rc;
     }
+    // Blocks of 2^15 are finished by one CTA each.  Up to 64 of them would leave
+    // more than half of the SMs idle during the longest kernel of the route: then
+    // one more level runs in HBM and twice as many CTAs finish blocks of 2^14.
+    const int fused_m = (T >> kFusedLog2M) <= 64 ? kFusedLog2M - 1 : kFusedLog2M;
     int cur = 0;
-    for (int level = 0; n - level > kFusedLog2M; ++level) {
+    for (int level = 0; n - level > fused_m; ++level) {
         const int m = n - level;
         const int out_stage = 2 * n - 2 - level;
         void *S = Sbuf[cur];
@@ -204,12 +208,12 @@ int route_levels(const uint32_t *perm, int n, size_t batch, uint32_t *bits, char
     }
     {
         ProfileScope ps(kFused, s);
-        if ((rc = launch_fused(Sbuf[cur], rec_is_packed(kFusedLog2M, kappa) ? 2 : 1, T, kFusedLog2M, bits, n, s))) return rc;
+        if ((rc = launch_fused(Sbuf[cur], rec_is_packed(fused_m, kappa) ? 2 : 1, T, fused_m, bits, n, s))) return rc;
     }
     if (hp && hp->bits_host) {
         // the stages of the in-CTA levels are one run of rows in the middle
-        const int first = n - kFusedLog2M;
-        if ((rc = copy_stage_rows(*hp, bits, n, batch, first, 2 * kFusedLog2M - 1, s))) return rc;
+        const int first = n - fused_m;
+        if ((rc = copy_stage_rows(*hp, bits, n, batch, first, 2 * fused_m - 1, s))) return rc;
     }
     return BENES_OK;
 }
