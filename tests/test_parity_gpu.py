@@ -310,6 +310,33 @@ def test_route_large_properties(n):
     binding.benes_release_workspace()
 
 
+def test_route_maximum_size_properties():
+    """N = 2^30, the largest size the ABI accepts (32-bit flat indices): same two
+    properties.  The permutation is drawn on the device (torch.randperm with a fixed
+    seed): the host generator would take minutes at this size, and no oracle value
+    is involved."""
+    n = 30
+    torch.manual_seed(30)
+    d_perm = torch.randperm(1 << n, device="cuda", dtype=torch.int32)
+    bits = torch.empty(binding.benes_switch_words(n, 1), dtype=torch.int32, device="cuda")
+    binding.benes_route(d_perm, n, 1, bits)
+    ident = torch.arange(1 << n, dtype=torch.int32, device="cuda")
+    out = torch.empty_like(ident)
+    binding.benes_apply_ex(bits, ident, out, 4, n, 1)
+    torch.cuda.synchronize()
+    assert torch.equal(out, d_perm)
+    del ident, out, d_perm
+    rows = bits.view(2 * n - 1, (1 << n) // 64)
+    for level in range(n - 1):
+        half = (1 << (n - level)) // 2                  # switches per block
+        first = torch.arange(1 << level, device="cuda", dtype=torch.int64) * half
+        words = rows[2 * n - 2 - level][first >> 5].to(torch.int64) & 0xFFFFFFFF
+        assert not bool(((words >> (first & 31)) & 1).any()), level
+    del rows, bits
+    binding.benes_release_workspace()
+    torch.cuda.empty_cache()
+
+
 # ---- host-buffer entry points, validation, robustness -------------------------------------------
 @pytest.mark.parametrize("n,batch,pinned", [(15, 2, False), (17, 3, False), (18, 1, True), (23, 1, True), (23, 1, False)])
 def test_host_entry_points(n, batch, pinned):
