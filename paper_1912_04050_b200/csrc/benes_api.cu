@@ -114,7 +114,7 @@ int copy_stage_rows(const HostPipe &hp, const uint32_t *bits, int n, size_t batc
     return BENES_OK;
 }
 
-// Levels 0 .. n-kFusedLog2M-1 in HBM, then the fused tail.
+// The levels whose blocks exceed the in-CTA size in HBM, then the fused tail.
 int route_levels(const uint32_t *perm, int n, size_t batch, uint32_t *bits, char *ws, cudaStream_t s,
                  const HostPipe *hp = nullptr) {
     const size_t T = batch << n;
