@@ -96,6 +96,7 @@ size_t apply_ws_bytes(int elem_bytes, int log2n, size_t batch) {
 // piece as soon as it is there), and the two stages a level has finished are
 // copied to the host on the side stream while the next levels run.
 constexpr int kMaxPieces = 8;
+constexpr int kFusedSplitWave = 148;   // CTAs of the fused kernel that run together (one per SM)
 struct HostPipe {
     uint32_t *bits_host = nullptr;     // finished stages go here (same layout as `bits`)
     cudaStream_t side = nullptr;
@@ -206,14 +207,40 @@ int route_levels(const uint32_t *perm, int n, size_t batch, uint32_t *bits, char
             if ((rc = copy_stage_rows(*hp, bits, n, batch, out_stage, 1, hp->side))) return rc;
         }
     }
+    const int records = rec_is_packed(fused_m, kappa) ? 2 : 1;
+    const size_t blocks = T >> fused_m;
+    // the stages of the in-CTA levels are one run of rows in the middle
+    const int first = n - fused_m, rows = 2 * fused_m - 1;
+    if (hp && hp->bits_host && batch == 1 && blocks >= 4 * size_t(kFusedSplitWave)) {
+        // Two launches of whole waves of CTAs (one CTA per SM): the columns the
+        // first one has finished go to the host while the second one runs.
+        const size_t waves = (blocks + kFusedSplitWave - 1) / kFusedSplitWave;
+        const size_t b1 = ((waves + 1) / 2) * kFusedSplitWave;
+        {
+            ProfileScope ps(kFused, s);
+            if ((rc = launch_fused(Sbuf[cur], records, T, fused_m, bits, n, s, 0, b1))) return rc;
+        }
+        BENES_CUDA_TRY(cudaEventRecord(hp->stage_ready[kMaxLevels - 2], s));
+        {
+            ProfileScope ps(kFused, s);
+            if ((rc = launch_fused(Sbuf[cur], records, T, fused_m, bits, n, s, b1, blocks - b1))) return rc;
+        }
+        // a block of 2^m outputs owns 2^(m-6) words of every stage
+        const size_t w = stage_words(n) * 4, col1 = (b1 << (fused_m - 6)) * 4;
+        char *dst = reinterpret_cast<char *>(hp->bits_host) + size_t(first) * w;
+        const char *src = reinterpret_cast<const char *>(bits) + size_t(first) * w;
+        BENES_CUDA_TRY(cudaStreamWaitEvent(hp->side, hp->stage_ready[kMaxLevels - 2], 0));
+        BENES_CUDA_TRY(cudaMemcpy2DAsync(dst, w, src, w, col1, size_t(rows), cudaMemcpyDeviceToHost, hp->side));
+        BENES_CUDA_TRY(cudaMemcpy2DAsync(dst + col1, w, src + col1, w, w - col1, size_t(rows),
+                                         cudaMemcpyDeviceToHost, s));
+        return BENES_OK;
+    }
     {
         ProfileScope ps(kFused, s);
-        if ((rc = launch_fused(Sbuf[cur], rec_is_packed(fused_m, kappa) ? 2 : 1, T, fused_m, bits, n, s))) return rc;
+        if ((rc = launch_fused(Sbuf[cur], records, T, fused_m, bits, n, s))) return rc;
     }
     if (hp && hp->bits_host) {
-        // the stages of the in-CTA levels are one run of rows in the middle
-        const int first = n - fused_m;
-        if ((rc = copy_stage_rows(*hp, bits, n, batch, first, 2 * fused_m - 1, s))) return rc;
+        if ((rc = copy_stage_rows(*hp, bits, n, batch, first, rows, s))) return rc;
     }
     return BENES_OK;
 }

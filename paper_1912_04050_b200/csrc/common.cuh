@@ -218,8 +218,9 @@ int sampled_scratch_reset(const SampledScratch &sc, size_t total, int kappa, cud
 // Finishes levels (n - log2m) .. n-1 of every block of size 2^log2m of the flat
 // level array (total elements), one CTA per block.  log2m <= kFusedLog2M.
 // P is a plain uint32 array if records == 0, wide records if 1, packed records if 2.
+// `blocks` blocks from `first_block` on (blocks = 0: all from first_block).
 int launch_fused(const void *P, int records, size_t total, int log2m, uint32_t *bits, int log2n,
-                 cudaStream_t s);
+                 cudaStream_t s, size_t first_block = 0, size_t blocks = 0);
 
 // ---- payload apply (apply.cu) ----------------------------------------------
 int launch_apply_stage(const uint32_t *bits, const void *x, void *y, int elem_bytes, int stage,

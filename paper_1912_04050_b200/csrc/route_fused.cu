@@ -50,7 +50,8 @@ __device__ __forceinline__ uint32_t fused_slot(uint32_t group, uint32_t salt) {
 
 template <int LOGM>
 __global__ void __launch_bounds__(FusedCfg<LOGM>::kThreads)
-k_route_fused(const uint32_t *__restrict__ P, int records, uint32_t *__restrict__ bits, int log2n) {
+k_route_fused(const uint32_t *__restrict__ P, int records, uint32_t *__restrict__ bits, int log2n,
+              uint32_t block0) {
     using C = FusedCfg<LOGM>;
     constexpr int M = C::M;
     constexpr int T = C::kThreads;
@@ -73,7 +74,7 @@ k_route_fused(const uint32_t *__restrict__ P, int records, uint32_t *__restrict_
     const int lane = tid & 31;
     const int n = log2n;
     const int level0 = n - LOGM;               // recursion level of this CTA's block
-    const size_t flat0 = size_t(blockIdx.x) << LOGM;
+    const size_t flat0 = size_t(blockIdx.x + block0) << LOGM;    // a launch may cover a range of the blocks
     // where this CTA's words of a stage start
     const size_t N = size_t(1) << n;
     const size_t stage_w = N >= 64 ? N / 64 : 1;
@@ -352,7 +353,8 @@ k_route_fused(const uint32_t *__restrict__ P, int records, uint32_t *__restrict_
 }
 
 template <int LOGM>
-int launch_one(const uint32_t *P, int records, size_t total, uint32_t *bits, int log2n, cudaStream_t s) {
+int launch_one(const uint32_t *P, int records, size_t first_block, size_t blocks, uint32_t *bits, int log2n,
+               cudaStream_t s) {
     using C = FusedCfg<LOGM>;
     static OncePerDevice configured;
     if (C::kSmemBytes > 48 * 1024 && configured.first_use()) {
@@ -363,32 +365,35 @@ int launch_one(const uint32_t *P, int records, size_t total, uint32_t *bits, int
                                             cudaFuncAttributePreferredSharedMemoryCarveout,
                                             cudaSharedmemCarveoutMaxShared));
     }
-    size_t blocks = total >> LOGM;
-    k_route_fused<LOGM><<<unsigned(blocks), C::kThreads, C::kSmemBytes, s>>>(P, records, bits, log2n);
+    k_route_fused<LOGM><<<unsigned(blocks), C::kThreads, C::kSmemBytes, s>>>(P, records, bits, log2n,
+                                                                             uint32_t(first_block));
     return launch_status();
 }
 
 }  // namespace
 
 int launch_fused(const void *Pv, int records, size_t total, int log2m, uint32_t *bits, int log2n,
-                 cudaStream_t s) {
+                 cudaStream_t s, size_t first_block, size_t blocks) {
     const uint32_t *P = static_cast<const uint32_t *>(Pv);
+    if (log2m < 1 || log2m > kFusedLog2M) return BENES_ERR_BADARG;
+    if (blocks == 0) blocks = (total >> log2m) - first_block;        // all the rest
+    if (first_block + blocks > (total >> log2m)) return BENES_ERR_BADARG;
     switch (log2m) {
-        case 1: return launch_one<1>(P, records, total, bits, log2n, s);
-        case 2: return launch_one<2>(P, records, total, bits, log2n, s);
-        case 3: return launch_one<3>(P, records, total, bits, log2n, s);
-        case 4: return launch_one<4>(P, records, total, bits, log2n, s);
-        case 5: return launch_one<5>(P, records, total, bits, log2n, s);
-        case 6: return launch_one<6>(P, records, total, bits, log2n, s);
-        case 7: return launch_one<7>(P, records, total, bits, log2n, s);
-        case 8: return launch_one<8>(P, records, total, bits, log2n, s);
-        case 9: return launch_one<9>(P, records, total, bits, log2n, s);
-        case 10: return launch_one<10>(P, records, total, bits, log2n, s);
-        case 11: return launch_one<11>(P, records, total, bits, log2n, s);
-        case 12: return launch_one<12>(P, records, total, bits, log2n, s);
-        case 13: return launch_one<13>(P, records, total, bits, log2n, s);
-        case 14: return launch_one<14>(P, records, total, bits, log2n, s);
-        case 15: return launch_one<15>(P, records, total, bits, log2n, s);
+        case 1: return launch_one<1>(P, records, first_block, blocks, bits, log2n, s);
+        case 2: return launch_one<2>(P, records, first_block, blocks, bits, log2n, s);
+        case 3: return launch_one<3>(P, records, first_block, blocks, bits, log2n, s);
+        case 4: return launch_one<4>(P, records, first_block, blocks, bits, log2n, s);
+        case 5: return launch_one<5>(P, records, first_block, blocks, bits, log2n, s);
+        case 6: return launch_one<6>(P, records, first_block, blocks, bits, log2n, s);
+        case 7: return launch_one<7>(P, records, first_block, blocks, bits, log2n, s);
+        case 8: return launch_one<8>(P, records, first_block, blocks, bits, log2n, s);
+        case 9: return launch_one<9>(P, records, first_block, blocks, bits, log2n, s);
+        case 10: return launch_one<10>(P, records, first_block, blocks, bits, log2n, s);
+        case 11: return launch_one<11>(P, records, first_block, blocks, bits, log2n, s);
+        case 12: return launch_one<12>(P, records, first_block, blocks, bits, log2n, s);
+        case 13: return launch_one<13>(P, records, first_block, blocks, bits, log2n, s);
+        case 14: return launch_one<14>(P, records, first_block, blocks, bits, log2n, s);
+        case 15: return launch_one<15>(P, records, first_block, blocks, bits, log2n, s);
         default: return BENES_ERR_BADARG;
     }
 }

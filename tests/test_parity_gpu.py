@@ -362,6 +362,21 @@ def test_host_entry_points(n, batch, pinned):
     assert np.array_equal(bits2, bits)
 
 
+def test_route_host_split_tail_matches_device_path():
+    """From 592 blocks of 2^15 on (N = 2^25 here) the host entry point finishes the
+    in-CTA levels in two launches and copies the first one's columns home while the
+    second runs.  Same words as the device entry point (whose result at this scale
+    is compared with the oracle in test_config4)."""
+    n = 25
+    perm = inputs.random_perm(n, 9)
+    want = gpu_route(perm, n)
+    perm_t = torch.from_numpy(perm.view(np.int32)).pin_memory()
+    bits_t = torch.full((2 * n - 1, (1 << n) // 64), 0x55555555, dtype=torch.int32).pin_memory()
+    binding.benes_route_host(perm_t, n, 1, bits_t)
+    assert np.array_equal(bits_t.numpy().view(np.uint32).reshape(want.shape), want)
+    binding.benes_release_workspace()
+
+
 def test_caller_workspace_is_used_and_checked():
     n = binding.benes_fused_log2m() + 2
     perm = inputs.random_perm(n, 11)
