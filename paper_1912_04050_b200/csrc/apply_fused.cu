@@ -161,10 +161,11 @@ __device__ __forceinline__ Geometry geometry(const uint32_t *bits, size_t flat, 
 // Inner kernel: all 2b-1 stages of one block of 2^b elements of level n-b.
 template <typename E>
 __global__ void __launch_bounds__(kApplyThreads, 2)
-k_apply_inner(const uint32_t *__restrict__ bits, const E *__restrict__ x, E *__restrict__ y, int n, int b) {
+k_apply_inner(const uint32_t *__restrict__ bits, const E *__restrict__ x, E *__restrict__ y, int n, int b,
+              uint32_t cta0) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     E *sm = reinterpret_cast<E *>(smem_raw);
-    const size_t flat0 = size_t(blockIdx.x) << b;
+    const size_t flat0 = size_t(blockIdx.x + cta0) << b;
     const Geometry g = geometry(bits, flat0, n, b);
     const int l0 = n - b;
     const uint32_t B = 1u << b;
@@ -193,10 +194,10 @@ k_apply_inner(const uint32_t *__restrict__ bits, const E *__restrict__ x, E *__r
 template <typename E, bool OUT>
 __global__ void __launch_bounds__(kApplyThreads, 3)
 k_apply_outer(const uint32_t *__restrict__ bits, const E *__restrict__ x, E *__restrict__ y, int n,
-              int l0, int k) {
+              int l0, int k, uint32_t cta0) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     E *sm = reinterpret_cast<E *>(smem_raw);
-    const size_t flat0 = size_t(blockIdx.x) << kChunkLog2;
+    const size_t flat0 = size_t(blockIdx.x + cta0) << kChunkLog2;
     const int m0 = n - l0;
     const Geometry g = geometry(bits, flat0, n, m0);
     const int tbits = kChunkLog2 - k;                               // log2 of the run length T
@@ -246,7 +247,7 @@ int opt_in_smem(K kernel, size_t bytes) {
 
 template <typename E>
 int apply_fused_typed(const uint32_t *bits, const E *in, E *out, E *scratch, int n, size_t batch,
-                      cudaStream_t s) {
+                      cudaStream_t s, const ApplyHostPipe *pipe) {
     const size_t total = batch << n;
     // payload slots + the switch words of up to 2*13-1 stages
     const size_t smem = size_t(kSmemElems) * sizeof(E) + size_t(2 * kChunkLog2 - 1) * kBitWords * 4;
@@ -273,12 +274,39 @@ int apply_fused_typed(const uint32_t *bits, const E *in, E *out, E *scratch, int
     int pass = 0;
     auto next_dst = [&]() { ++pass; return ((passes - pass) % 2 == 0) ? out : scratch; };
     const unsigned chunks = unsigned(total >> kChunkLog2);
-    int l0 = 0;
+    // A pass is one launch, or `parts` launches over equal ranges of CTAs: the
+    // first pass of a piped call waits for each part of `in`, its last pass
+    // hands each finished part of `out` to the side stream.  CTA c of the first
+    // (last) pass reads (writes) elements [c, c+1) * 2^13 (2^b in the inner pass).
+    const int total_passes = passes;
+    auto run_pass = [&](int index, unsigned ctas, size_t elems_per_cta, auto &&launch) -> int {
+        const bool first = pipe && index == 0, last = pipe && index == total_passes - 1;
+        const unsigned parts = (first || last) ? unsigned(pipe->parts) : 1u;
+        const unsigned per = ctas / parts;
+        for (unsigned p = 0; p < parts; ++p) {
+            if (first) BENES_CUDA_TRY(cudaStreamWaitEvent(s, pipe->in_ready[p], 0));
+            launch(per, p * per);
+            int rc = launch_status();
+            if (rc) return rc;
+            if (last) {
+                BENES_CUDA_TRY(cudaEventRecord(pipe->out_done[p], s));
+                BENES_CUDA_TRY(cudaStreamWaitEvent(pipe->side, pipe->out_done[p], 0));
+                const size_t off = size_t(p) * per * elems_per_cta * sizeof(E), bytes = size_t(per) * elems_per_cta * sizeof(E);
+                BENES_CUDA_TRY(cudaMemcpyAsync(static_cast<char *>(pipe->out_host) + off,
+                                               reinterpret_cast<const char *>(out) + off, bytes,
+                                               cudaMemcpyDeviceToHost, pipe->side));
+            }
+        }
+        return BENES_OK;
+    };
+    int l0 = 0, index = 0, rc;
     for (int i = 0; i < per_side; ++i) {
         E *dst = next_dst();
-        k_apply_outer<E, false><<<chunks, kApplyThreads, smem_outer, s>>>(bits, src, dst, n, l0, ks[i]);
-        int rc = launch_status();
-        if (rc) return rc;
+        const int k = ks[i], lvl = l0;
+        if ((rc = run_pass(index++, chunks, size_t(kChunk), [&](unsigned ctas, unsigned cta0) {
+                 k_apply_outer<E, false><<<ctas, kApplyThreads, smem_outer, s>>>(bits, src, dst, n, lvl, k, cta0);
+             })))
+            return rc;
         src = dst;
         l0 += ks[i];
     }
@@ -287,17 +315,20 @@ int apply_fused_typed(const uint32_t *bits, const E *in, E *out, E *scratch, int
         const unsigned blocks = unsigned(total >> b);
         unsigned threads = (1u << b) >> kRound;
         threads = threads < 32u ? 32u : (threads > unsigned(kApplyThreads) ? unsigned(kApplyThreads) : threads);
-        k_apply_inner<E><<<blocks, threads, smem, s>>>(bits, src, dst, n, b);
-        int rc = launch_status();
-        if (rc) return rc;
+        if ((rc = run_pass(index++, blocks, size_t(1) << b, [&](unsigned ctas, unsigned cta0) {
+                 k_apply_inner<E><<<ctas, threads, smem, s>>>(bits, src, dst, n, b, cta0);
+             })))
+            return rc;
         src = dst;
     }
     for (int i = per_side - 1; i >= 0; --i) {
         E *dst = next_dst();
         l0 -= ks[i];
-        k_apply_outer<E, true><<<chunks, kApplyThreads, smem_outer, s>>>(bits, src, dst, n, l0, ks[i]);
-        int rc = launch_status();
-        if (rc) return rc;
+        const int k = ks[i], lvl = l0;
+        if ((rc = run_pass(index++, chunks, size_t(kChunk), [&](unsigned ctas, unsigned cta0) {
+                 k_apply_outer<E, true><<<ctas, kApplyThreads, smem_outer, s>>>(bits, src, dst, n, lvl, k, cta0);
+             })))
+            return rc;
         src = dst;
     }
     return BENES_OK;
@@ -310,17 +341,24 @@ int apply_fused_passes(int log2n) {
     return 2 * ((log2n - b + 6) / 7) + 1;
 }
 
+size_t apply_fused_chunks(int log2n, size_t batch) {
+    return log2n > kChunkLog2 ? (batch << log2n) >> kChunkLog2 : 0;
+}
+
 int launch_apply_fused(const uint32_t *bits, const void *in, void *out, void *scratch, int elem_bytes,
-                       int log2n, size_t batch, cudaStream_t s) {
+                       int log2n, size_t batch, cudaStream_t s, const ApplyHostPipe *pipe) {
+    if (pipe && (pipe->parts < 1 || pipe->parts > kApplyMaxParts ||
+                 apply_fused_chunks(log2n, batch) % size_t(pipe->parts) != 0 || apply_fused_chunks(log2n, batch) == 0))
+        return BENES_ERR_BADARG;
     if (elem_bytes == 4)
         return apply_fused_typed<uint32_t>(bits, static_cast<const uint32_t *>(in),
                                            static_cast<uint32_t *>(out), static_cast<uint32_t *>(scratch),
-                                           log2n, batch, s);
+                                           log2n, batch, s, pipe);
     if (elem_bytes == 8)
         return apply_fused_typed<unsigned long long>(bits, static_cast<const unsigned long long *>(in),
                                                      static_cast<unsigned long long *>(out),
                                                      static_cast<unsigned long long *>(scratch), log2n,
-                                                     batch, s);
+                                                     batch, s, pipe);
     return BENES_ERR_BADARG;
 }
 

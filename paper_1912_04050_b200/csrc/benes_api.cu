@@ -96,6 +96,7 @@ size_t apply_ws_bytes(int elem_bytes, int log2n, size_t batch) {
 // piece as soon as it is there), and the two stages a level has finished are
 // copied to the host on the side stream while the next levels run.
 constexpr int kMaxPieces = 8;
+static_assert(kMaxPieces >= kApplyMaxParts, "the host pipe's events serve the apply parts too");
 constexpr int kFusedSplitWave = 148;   // CTAs of the fused kernel that run together (one per SM)
 struct HostPipe {
     uint32_t *bits_host = nullptr;     // finished stages go here (same layout as `bits`)
@@ -486,6 +487,36 @@ int benes_apply_host(const uint32_t *switch_bits_host, const void *in_host, void
     char *d_out = d_in + align_up(data_bytes);
     uint32_t *d_bits = reinterpret_cast<uint32_t *>(d_out + align_up(data_bytes));
     BENES_CUDA_TRY(cudaMemcpyAsync(d_bits, switch_bits_host, bits_bytes, cudaMemcpyHostToDevice, s));
+    const size_t chunks = apply_fused_chunks(log2n, size_t(batch));
+    if (g_apply_fused && data_bytes >= (size_t(1) << 26) && chunks % kApplyMaxParts == 0 && chunks > 0) {
+        // The payload arrives in parts on the side stream, behind the switch words:
+        // the first pass starts on a part as soon as it is there, and the parts the
+        // last pass has finished leave on the side stream while it still runs.
+        HostPipe *hp = nullptr;
+        if ((rc = host_pipe_for_current_device(&hp))) return rc;
+        ApplyHostPipe pipe;
+        pipe.parts = kApplyMaxParts;
+        pipe.side = hp->side;
+        pipe.out_host = out_host;
+        // the side stream must not touch the workspace before earlier work on `s` is done
+        BENES_CUDA_TRY(cudaEventRecord(hp->stage_ready[kMaxLevels - 1], s));
+        BENES_CUDA_TRY(cudaStreamWaitEvent(hp->side, hp->stage_ready[kMaxLevels - 1], 0));
+        const size_t per = data_bytes / size_t(pipe.parts);
+        for (int i = 0; i < pipe.parts; ++i) {
+            pipe.in_ready[i] = hp->piece_ready[i];
+            pipe.out_done[i] = hp->stage_ready[i];
+            BENES_CUDA_TRY(cudaMemcpyAsync(d_in + per * size_t(i), static_cast<const char *>(in_host) + per * size_t(i),
+                                           per, cudaMemcpyHostToDevice, hp->side));
+            BENES_CUDA_TRY(cudaEventRecord(hp->piece_ready[i], hp->side));
+        }
+        {
+            ProfileScope ps(kApplyFused, s);
+            rc = launch_apply_fused(d_bits, d_in, d_out, base, elem_bytes, log2n, size_t(batch), s, &pipe);
+        }
+        cudaError_t e1 = cudaStreamSynchronize(s), e2 = cudaStreamSynchronize(hp->side);
+        if (rc) return rc;
+        return (e1 == cudaSuccess && e2 == cudaSuccess) ? BENES_OK : BENES_ERR_CUDA;
+    }
     BENES_CUDA_TRY(cudaMemcpyAsync(d_in, in_host, data_bytes, cudaMemcpyHostToDevice, s));
     rc = benes_apply_ex(d_bits, d_in, d_out, elem_bytes, log2n, batch, stream);
     if (rc) return rc;

@@ -229,8 +229,21 @@ int launch_apply_stage(const uint32_t *bits, const void *x, void *y, int elem_by
 // ---- payload apply, several stages per pass (apply_fused.cu) -----------------
 // `scratch` (batch * N elements) is needed when apply_fused_passes(log2n) > 1.
 int apply_fused_passes(int log2n);
+// With a pipe the first pass runs part by part as the parts of `in` arrive
+// (in_ready[i], recorded on another stream), and the parts of `out` the last
+// pass has finished are copied to out_host on the side stream.
+constexpr int kApplyMaxParts = 8;
+struct ApplyHostPipe {
+    int parts;                              // divides the number of 2^13-element chunks
+    cudaEvent_t in_ready[kApplyMaxParts];
+    cudaEvent_t out_done[kApplyMaxParts];
+    cudaStream_t side;
+    void *out_host;
+};
 int launch_apply_fused(const uint32_t *bits, const void *in, void *out, void *scratch, int elem_bytes,
-                       int log2n, size_t batch, cudaStream_t s);
+                       int log2n, size_t batch, cudaStream_t s, const ApplyHostPipe *pipe = nullptr);
+// chunks (CTAs) of the first and of the last pass, 0 if the size is too small to pipe
+size_t apply_fused_chunks(int log2n, size_t batch);
 
 // ---- sizes that are not a power of two (pad.cu) ------------------------------
 int launch_pad_perm(const uint32_t *src, uint32_t *dst, size_t n_elems, int log2n, size_t batch,

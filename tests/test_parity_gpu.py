@@ -377,6 +377,19 @@ def test_route_host_split_tail_matches_device_path():
     binding.benes_release_workspace()
 
 
+def test_apply_host_piped_u32():
+    """Payloads of 64 MiB and more go through benes_apply_host in parts (first pass
+    as the parts arrive, last pass handing finished parts to the copy stream)."""
+    n = 24
+    perm = inputs.random_perm(n, 13)
+    bits = gpu_route(perm, n)
+    x = inputs.payload_u64(1 << (n - 1), 6).view(np.uint32).copy()
+    out = np.full_like(x, 0xDEADBEEF)
+    binding.benes_apply_host(bits, x, out, 4, n, 1)
+    assert np.array_equal(out, x[perm.astype(np.int64)])
+    binding.benes_release_workspace()
+
+
 def test_caller_workspace_is_used_and_checked():
     n = binding.benes_fused_log2m() + 2
     perm = inputs.random_perm(n, 11)
