@@ -143,10 +143,13 @@ int benes_apply_static(const uint32_t *switch_bits, const void *in, void *out, i
  * Host-buffer variants: copy the inputs to the device, run, copy the result
  * back and SYNCHRONISE `stream` before returning.  Buffers are ordinary or
  * pinned host memory (pinned memory lets the copies overlap the kernels).
- * Device staging lives in the library workspace.  benes_route_host overlaps
- * its copies with the computation on a second stream the library owns (one per
- * device, created on the first call): the permutation arrives in pieces, and
- * the stages a level has finished go back while the next levels run.
+ * Device staging lives in the library workspace.  Both calls overlap their
+ * copies with the computation on a second stream the library owns (one per
+ * device, created on the first call).  benes_route_host: the permutation
+ * arrives in pieces, and the stages a level has finished go back while the next
+ * levels run.  benes_apply_host (payloads of 64 MiB and more): the first pass
+ * starts on each part of the payload as it arrives, and the parts the last
+ * pass has finished go back while it still runs.
  */
 int benes_route_host(const uint32_t *perm_host, int log2n, int batch, uint32_t *switch_bits_host,
                      benes_stream_t stream);
