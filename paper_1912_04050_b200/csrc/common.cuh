@@ -200,6 +200,7 @@ int launch_split(const void *S, bool packed, const uint32_t *Q, void *Sn, bool n
 // ---- ruler-sampled loop labelling (route_sampled.cu) --------------------------
 struct SampledScratch {
     uint4 *rec;                  // total >> kappa walk records
+    uint32_t *ruler_bits;        // parity of every ruler's cycle minimum, one bit each
     unsigned long long *list[5]; // contracted lists: total >> (kappa + 4 i) words
     uint32_t *owner[5];          // owners of the words of list[i] (all kUnowned between uses)
 };

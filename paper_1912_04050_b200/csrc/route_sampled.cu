@@ -289,6 +289,60 @@ int launch_list_label(unsigned long long *W, uint32_t count, int beta, uint32_t 
     return launch_status();
 }
 
+// Steps 3 and 4 in one kernel for a level whose blocks have at most 2^18 outputs
+// and lists that fit one CTA (no sampling of the list): the CTA forms its
+// block's list words from the walk records, (next, min) = (peer ^ 1,
+// min(fwd[rho], part[peer])), as 14 + 18 bit, both local to the block, labels
+// them by synchronous pointer jumping and writes the parity bits.  Indices a
+// raised gate may have left undefined are masked into the block.
+template <int PER>
+__global__ void __launch_bounds__(kListThreads)
+k_list_label_rec(const uint4 *__restrict__ rec, uint32_t *__restrict__ cb, int log2b, int m) {
+    extern __shared__ uint32_t sw[];
+    constexpr uint32_t kNext = (1u << kListSmemLog2) - 1u;
+    const uint32_t B = 1u << log2b, bmask = B - 1u, mmask = (1u << m) - 1u;
+    const uint32_t base = blockIdx.x << log2b;                    // first ruler output of the block
+    const uint32_t T = blockDim.x, tid = threadIdx.x;
+#pragma unroll
+    for (int i = 0; i < PER; ++i) {
+        const uint32_t e = tid + uint32_t(i) * T;
+        const uint4 a = __ldcs(rec + base + e);
+        const uint32_t peer = a.z & bmask;
+        const uint4 b = __ldg(rec + base + peer);
+        sw[e] = (peer ^ 1u) | ((min(a.x, b.y) & mmask) << kListSmemLog2);
+    }
+    __syncthreads();
+    uint32_t v[PER];
+    for (int pass = 0; pass < log2b; ++pass) {
+#pragma unroll
+        for (int i = 0; i < PER; ++i) {
+            const uint32_t w = sw[tid + uint32_t(i) * T];
+            const uint32_t t = sw[w & kNext];
+            v[i] = (t & kNext) | min(w & ~kNext, t & ~kNext);
+        }
+        __syncthreads();
+#pragma unroll
+        for (int i = 0; i < PER; ++i) sw[tid + uint32_t(i) * T] = v[i];
+        __syncthreads();
+    }
+#pragma unroll
+    for (int i = 0; i < PER; ++i) {
+        const uint32_t e = tid + uint32_t(i) * T;
+        const uint32_t word = __ballot_sync(0xFFFFFFFFu, (sw[e] >> kListSmemLog2) & 1u);
+        if ((tid & 31u) == 0u) cb[(base + e) >> 5] = word;
+    }
+}
+
+template <int PER>
+int launch_list_label_rec(const uint4 *rec, uint32_t *cb, uint32_t count, int beta, int m, cudaStream_t s) {
+    static OncePerDevice configured;
+    if (configured.first_use())
+        BENES_CUDA_TRY(cudaFuncSetAttribute(k_list_label_rec<PER>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            (1 << kListSmemLog2) * 4));
+    k_list_label_rec<PER><<<count >> beta, (1u << beta) / PER, (size_t(1) << beta) * 4, s>>>(rec, cb, beta, m);
+    return launch_status();
+}
+
 // Step 5: colour of output 2t from the owner of switch t, or by walking the cycle.
 template <bool PACKED>
 __device__ __forceinline__ uint32_t colour_of(const void *S, const uint32_t *Q, const uint32_t *cb,
@@ -454,7 +508,7 @@ inline int list_depth(int beta) {
 // Scratch: walk records, the contracted lists and the owners of every list
 // that may be sampled again.  Sized for the largest level (log2m = 30).
 size_t sampled_scratch_bytes(size_t total, int kappa) {
-    size_t R = total >> kappa, bytes = align256(R * 16);
+    size_t R = total >> kappa, bytes = align256(R * 16) + align256(R / 8 + 4);
     for (int i = 0; i < kMaxLists; ++i) {
         size_t c = R >> (kListKappa * i);
         if (c < 4) c = 4;
@@ -467,6 +521,8 @@ void sampled_scratch_carve(char *base, size_t total, int kappa, SampledScratch *
     size_t R = total >> kappa, off = 0;
     out->rec = reinterpret_cast<uint4 *>(base);
     off += align256(R * 16);
+    out->ruler_bits = reinterpret_cast<uint32_t *>(base + off);
+    off += align256(R / 8 + 4);
     for (int i = 0; i < kMaxLists; ++i) {
         size_t c = R >> (kListKappa * i);
         if (c < 4) c = 4;
@@ -500,18 +556,26 @@ int sampled_label(void *S, bool packed, const uint32_t *Q, void *Sn, bool next_p
         int rc = launch_status();
         if (rc) return rc;
     }
-    {
+    uint32_t *cb = sc.ruler_bits;
+    // label the contracted list: sample it until a block's list fits one CTA
+    int beta = log2m - kappa;
+    const int depth = list_depth(beta);
+    uint32_t count = R;
+    // (the kernels that write the parity bits ballot: whole warps, i.e. lists of 2^7 words at least)
+    if (depth == 0 && beta < 7) return BENES_ERR_BADARG;
+    const bool from_records = depth == 0 && log2m <= 32 - kListSmemLog2;
+    if (from_records) {
+        ProfileScope ps(kListLabel, s);
+        int rc = beta <= 12 ? launch_list_label_rec<4>(sc.rec, cb, count, beta, log2m, s)
+               : beta == 13 ? launch_list_label_rec<8>(sc.rec, cb, count, beta, log2m, s)
+                            : launch_list_label_rec<16>(sc.rec, cb, count, beta, log2m, s);
+        if (rc) return rc;
+    } else {
         ProfileScope ps(kCombine, s);
         k_combine<<<rgrid, kThreads, 0, s>>>(sc.rec, sc.list[0], R);
         int rc = launch_status();
         if (rc) return rc;
     }
-    // the walk records are dead: their memory takes the rulers' colour bits
-    uint32_t *cb = reinterpret_cast<uint32_t *>(sc.rec);
-    // label the contracted list: sample it until a block's list fits one CTA
-    int beta = log2m - kappa;
-    const int depth = list_depth(beta);
-    uint32_t count = R;
     for (int d = 0; d < depth; ++d) {
         ProfileScope ps(kListWalk, s);
         const uint32_t next = count >> kListKappa;
@@ -523,7 +587,7 @@ int sampled_label(void *S, bool packed, const uint32_t *Q, void *Sn, bool next_p
         count = next;
         beta -= kListKappa;
     }
-    {
+    if (!from_records) {
         ProfileScope ps(kListLabel, s);
         if (beta > kListSmemLog2 || beta < 5) return BENES_ERR_BADARG;
         // 4 words per thread up to 2^12 words, then 1024 threads
