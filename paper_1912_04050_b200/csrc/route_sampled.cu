@@ -22,8 +22,9 @@
 //      per ruler output -- the contracted list.
 //   4. The contracted list is labelled with the minimum of every cycle:
 //      lists of up to 2^14 words per block in one CTA's shared memory, longer
-//      ones by sampling again (one ruler per 16 words, plain one-directional
-//      walks: the list is cache resident).
+//      ones by sampling again: the list is mirror symmetric like the loops, so
+//      it is sampled the same way (one ruler pair per 16 pairs of words, walks
+//      that meet in the middle, k_combine again).
 //   5. k_colour: output 2t lies on its owner's cycle if the owner arrived on
 //      the even side, else on the mirror cycle, which has the other colour:
 //      colour = (cycle minimum of the owner & 1) ^ side.  A switch nobody
@@ -155,25 +156,35 @@ k_combine(const uint4 *__restrict__ rec, unsigned long long *__restrict__ W, uin
     W[rho] = make_word(peer ^ 1u, min(a.x, b.y));
 }
 
-// Step 4, sampling a list: one ruler per 16 words; a thread walks from its
-// ruler to the next one, stamps itself on the words it passes and writes one
-// word (next ruler, minimum) of the 16 times shorter list.
-__global__ void __launch_bounds__(kThreads)
-k_list_walk(const unsigned long long *__restrict__ W, uint32_t *__restrict__ owner,
-            unsigned long long *__restrict__ W2, uint32_t rulers, uint32_t wmask, uint32_t salt,
-            uint32_t cap, uint32_t *__restrict__ gate) {
-    const uint32_t rho = blockIdx.x * kThreads + threadIdx.x;
-    if (rho >= rulers) return;
-    constexpr uint32_t kmask = (1u << kListKappa) - 1u;
-    uint32_t e = (rho << kListKappa) | ruler_slot(rho, salt, kmask);
-    unsigned long long w = __ldcg(W + e);
-    uint32_t mn = uint32_t(w >> 32), nxt = rho, hops = 0;
-    owner[e] = rho;
+// Step 4, sampling a list.  The contracted list inherits the mirror symmetry
+// of the loops (next[rho] = sigma implies next[sigma ^ 1] = rho ^ 1), and so does
+// every list sampled from it this way: a list is sampled the way the switches are.  Words 2q and 2q+1 form a pair; one pair per 16
+// pairs is a ruler pair, both of its words start a walker; the walker from the
+// even word runs along its cycle, the walker from the odd word of the NEXT
+// ruler pair runs along the mirror cycle, i.e. over the same pairs from the
+// other end; each claims pairs (owner[q] = walker, side of arrival) and stops
+// where the other one has been.  The longest walk of a launch is half as long
+// as with one-directional walks.  A walker keeps the minimum over the words it
+// passed (fwd), over their partners (part) and whom it met (peer): the same
+// record as in step 2, turned into the 16 times shorter list by k_combine.
+constexpr int kPairGroupLog2 = kListKappa;          // pairs per ruler pair (log2)
+
+__global__ void __launch_bounds__(kWalkThreads)
+k_list_walk_pairs(const ulonglong2 *__restrict__ W2p, uint32_t *__restrict__ owner, uint4 *__restrict__ rec,
+                  uint32_t rulers, uint32_t pmask, uint32_t salt, uint32_t cap, uint32_t *__restrict__ gate) {
+    const uint32_t sigma = blockIdx.x * kWalkThreads + threadIdx.x;
+    if (sigma >= rulers) return;
+    constexpr uint32_t kmask = (1u << kPairGroupLog2) - 1u;
+    const uint32_t group = sigma >> 1, side0 = sigma & 1u;
+    const uint32_t q0 = (group << kPairGroupLog2) | ruler_slot(group, salt, kmask);
+    ulonglong2 w = __ldcg(W2p + q0);
+    if (!side0) owner[q0] = sigma << 1;                            // the ruler pair belongs to its even walker
+    unsigned long long own = side0 ? w.y : w.x;
+    uint32_t fwd = uint32_t(own >> 32), part = kUnowned, peer = sigma ^ 1u, hops = 0;
     for (;;) {
-        e = uint32_t(w) & wmask;
-        const uint32_t g = e >> kListKappa;
-        if ((e & kmask) == ruler_slot(g, salt, kmask)) {
-            nxt = g;
+        const uint32_t e = uint32_t(own), q = (e >> 1) & pmask, side = e & 1u, g = q >> kPairGroupLog2;
+        if ((q & kmask) == ruler_slot(g, salt, kmask)) {           // reached the next ruler pair
+            peer = (2u * g + side) ^ 1u;
             break;
         }
         if (++hops > cap) {
@@ -181,52 +192,80 @@ k_list_walk(const unsigned long long *__restrict__ W, uint32_t *__restrict__ own
             break;
         }
         if ((hops & 63u) == 0u && gate_raised(gate)) break;
-        w = __ldcg(W + e);
-        mn = min(mn, uint32_t(w >> 32));
-        owner[e] = rho;
+        w = __ldcg(W2p + q);
+        const uint32_t prev = atomicCAS(owner + q, kUnowned, (sigma << 1) | side);
+        if (prev != kUnowned) {                                    // met the walker from the other end
+            peer = prev >> 1;
+            break;
+        }
+        own = side ? w.y : w.x;
+        const unsigned long long far = side ? w.x : w.y;
+        fwd = min(fwd, uint32_t(own >> 32));
+        part = min(part, uint32_t(far >> 32));
     }
-    W2[rho] = make_word(nxt, mn);
+    rec[sigma] = make_uint4(fwd, part, peer, 0u);
 }
 
-// Step 4, back from a sampled list: every word takes the cycle minimum of its
-// owner (and hands the owner slot back as kUnowned); a word without owner
-// walks its own cycle.  For the first list (the rulers of the level) only the
-// parity of the minimum is needed afterwards: with `cb` the kernel writes one
-// bit per word there and leaves the words alone, so that the colouring kernel
-// gathers from an array 64 times smaller than the list (it stays in L1/L2 next
-// to the streaming traffic).  count is a multiple of 32.
-__global__ void __launch_bounds__(kThreads)
-k_list_resolve(unsigned long long *__restrict__ W, uint32_t *__restrict__ owner,
-               const unsigned long long *__restrict__ W2, uint32_t count, uint32_t wmask,
-               uint32_t cap, uint32_t *__restrict__ gate, uint32_t *__restrict__ cb) {
-    const uint32_t e0 = blockIdx.x * kThreads + threadIdx.x;
-    if (e0 >= count) return;
-    const uint32_t o = owner[e0];
-    unsigned long long w = __ldcg(W + e0);
-    uint32_t mn;
-    if (o != kUnowned) {
-        mn = uint32_t(__ldcg(W2 + o) >> 32);
-        owner[e0] = kUnowned;
-    } else {
-        // words rewritten meanwhile hold the minimum of this same cycle: harmless
-        mn = uint32_t(w >> 32);
-        uint32_t e = uint32_t(w) & wmask, hops = 0;
-        while (e != e0) {
-            if (++hops > cap) {
-                *gate = 1u;
-                break;
-            }
-            const unsigned long long v = __ldcg(W + e);
-            mn = min(mn, uint32_t(v >> 32));
-            e = uint32_t(v) & wmask;
+// Back from a sampled list: a thread takes the pair 2q, 2q+1 (and hands the
+// owner slot back as kUnowned).  Word 2q + b lies on its owner's cycle if the
+// owner arrived on side b, else on the mirror cycle, which is the cycle of the
+// owner's partner walker and whose minimum has the other parity.  A pair nobody
+// claimed lies on a cycle without ruler pair: the thread walks the cycle of
+// word 2q (and that of word 2q+1 if the minima themselves are needed).
+// Of the first list (the rulers of the level) only the parity of the minima is
+// needed afterwards: with `cb` one bit per word goes there, so that the colouring
+// kernel gathers from an array 64 times smaller than the list (it stays in
+// L1/L2 next to the streaming traffic); without, the words take their minima.
+__device__ __forceinline__ uint32_t list_cycle_min(const unsigned long long *W, uint32_t e0, uint32_t wmask,
+                                                   uint32_t cap, uint32_t *gate) {
+    unsigned long long v = __ldcg(W + e0);
+    uint32_t mn = uint32_t(v >> 32), e = uint32_t(v) & wmask, hops = 0;
+    while (e != e0) {
+        if (++hops > cap) {
+            *gate = 1u;
+            break;
         }
+        v = __ldcg(W + e);
+        mn = min(mn, uint32_t(v >> 32));       // words rewritten meanwhile hold the minimum of this same cycle
+        e = uint32_t(v) & wmask;
     }
-    if (cb) {
-        const uint32_t word = __ballot_sync(0xFFFFFFFFu, mn & 1u);
-        if ((threadIdx.x & 31) == 0) cb[e0 >> 5] = word;
+    return mn;
+}
+
+__global__ void __launch_bounds__(kThreads)
+k_list_resolve_pairs(unsigned long long *__restrict__ W, uint32_t *__restrict__ owner,
+                     const unsigned long long *__restrict__ W2, uint32_t pairs, uint32_t wmask,
+                     uint32_t cap, uint32_t *__restrict__ gate, uint32_t *__restrict__ cb) {
+    const uint32_t q = blockIdx.x * kThreads + threadIdx.x;       // pairs is a multiple of 32
+    if (q >= pairs) return;
+    const uint32_t code = owner[q];
+    if (!cb) {
+        uint32_t mn0, mn1;
+        if (code != kUnowned) {
+            const uint32_t a = uint32_t(__ldcg(W2 + (code >> 1)) >> 32), b = uint32_t(__ldcg(W2 + ((code >> 1) ^ 1u)) >> 32);
+            mn0 = (code & 1u) ? b : a;
+            mn1 = (code & 1u) ? a : b;
+            owner[q] = kUnowned;
+        } else {
+            mn0 = list_cycle_min(W, 2u * q, wmask, cap, gate);
+            mn1 = list_cycle_min(W, 2u * q + 1u, wmask, cap, gate);
+        }
+        ulonglong2 *Wp = reinterpret_cast<ulonglong2 *>(W) + q;
+        ulonglong2 w = *Wp;
+        w.x = make_word(uint32_t(w.x), mn0);
+        w.y = make_word(uint32_t(w.y), mn1);
+        *Wp = w;
+        return;
+    }
+    uint32_t bit0;
+    if (code != kUnowned) {
+        bit0 = (uint32_t(__ldcg(W2 + (code >> 1)) >> 32) ^ code) & 1u;
+        owner[q] = kUnowned;
     } else {
-        __stcg(W + e0, make_word(uint32_t(w), mn));
+        bit0 = list_cycle_min(W, 2u * q, wmask, cap, gate) & 1u;
     }
+    // a warp covers 64 words: two words of cb
+    store_stage_bits64(cb + ((q - (threadIdx.x & 31u)) >> 4), bit0, bit0 ^ 1u);
 }
 
 // Step 4, the end of the recursion: one CTA labels one block's list of
@@ -577,13 +616,23 @@ int sampled_label(void *S, bool packed, const uint32_t *Q, void *Sn, bool next_p
         if (rc) return rc;
     }
     for (int d = 0; d < depth; ++d) {
-        ProfileScope ps(kListWalk, s);
+        // walks from both ends; the walk records of the previous stage (switches,
+        // or the list before) are dead, their memory takes the new ones
         const uint32_t next = count >> kListKappa;
-        k_list_walk<<<(next + kThreads - 1) / kThreads, kThreads, 0, s>>>(
-            sc.list[d], sc.owner[d], sc.list[d + 1], next, count - 1u, salt * 7u + uint32_t(d) + 1u,
-            cap, gate);
-        int rc = launch_status();
-        if (rc) return rc;
+        {
+            ProfileScope ps(kListWalk, s);
+            k_list_walk_pairs<<<(next + kWalkThreads - 1) / kWalkThreads, kWalkThreads, 0, s>>>(
+                reinterpret_cast<const ulonglong2 *>(sc.list[d]), sc.owner[d], sc.rec, next, (count >> 1) - 1u,
+                salt * 7u + uint32_t(d) + 1u, cap, gate);
+            int rc = launch_status();
+            if (rc) return rc;
+        }
+        {
+            ProfileScope ps(kCombine, s);
+            k_combine<<<(next + kThreads - 1) / kThreads, kThreads, 0, s>>>(sc.rec, sc.list[d + 1], next);
+            int rc = launch_status();
+            if (rc) return rc;
+        }
         count = next;
         beta -= kListKappa;
     }
@@ -600,8 +649,8 @@ int sampled_label(void *S, bool packed, const uint32_t *Q, void *Sn, bool next_p
     for (int d = depth - 1; d >= 0; --d) {
         ProfileScope ps(kListResolve, s);
         const uint32_t c = R >> (kListKappa * d);
-        k_list_resolve<<<(c + kThreads - 1) / kThreads, kThreads, 0, s>>>(
-            sc.list[d], sc.owner[d], sc.list[d + 1], c, c - 1u, cap, gate, d == 0 ? cb : nullptr);
+        k_list_resolve_pairs<<<(c / 2 + kThreads - 1) / kThreads, kThreads, 0, s>>>(
+            sc.list[d], sc.owner[d], sc.list[d + 1], c / 2, c - 1u, cap, gate, d == 0 ? cb : nullptr);
         int rc = launch_status();
         if (rc) return rc;
     }
