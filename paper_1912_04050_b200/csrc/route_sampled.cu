@@ -271,9 +271,9 @@ k_list_resolve_pairs(unsigned long long *__restrict__ W, uint32_t *__restrict__ 
 // Step 4, the end of the recursion: one CTA labels one block's list of
 // 2^log2b words in shared memory by synchronous pointer jumping (new words are
 // held in registers across the barrier; PER words per thread, blockDim =
-// 2^log2b / PER).  A cycle has at most 2^log2b words (a list sampled from a
-// list need not split evenly between a cycle and its mirror image), hence
-// log2b passes.
+// 2^log2b / PER).  A cycle and its mirror image have the same number of words
+// and lie in the same block, so a cycle has at most 2^(log2b-1) words: log2b - 1
+// passes.
 // With `cb` (first list of a level) the parities of the minima go there, one bit
 // per word, instead of the words back to W.
 template <int PER>
@@ -291,7 +291,7 @@ k_list_label(unsigned long long *__restrict__ W, int log2b, uint32_t *__restrict
     }
     __syncthreads();
     unsigned long long v[PER];
-    for (int pass = 0; pass < log2b; ++pass) {
+    for (int pass = 0; pass < log2b - 1; ++pass) {
 #pragma unroll
         for (int i = 0; i < PER; ++i) {
             const unsigned long long w = sm[tid + uint32_t(i) * T];
@@ -352,7 +352,7 @@ k_list_label_rec(const uint4 *__restrict__ rec, uint32_t *__restrict__ cb, int l
     }
     __syncthreads();
     uint32_t v[PER];
-    for (int pass = 0; pass < log2b; ++pass) {
+    for (int pass = 0; pass < log2b - 1; ++pass) {
 #pragma unroll
         for (int i = 0; i < PER; ++i) {
             const uint32_t w = sw[tid + uint32_t(i) * T];
