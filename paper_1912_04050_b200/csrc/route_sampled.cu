@@ -382,63 +382,44 @@ int launch_list_label_rec(const uint4 *rec, uint32_t *cb, uint32_t count, int be
     return launch_status();
 }
 
-// Step 5: colour of output 2t from the owner of switch t, or by walking the cycle.
+// Step 5 for a switch on a loop without ruler: the minimum of the g-cycle C of
+// output 2t, walked from both ends.  The cycle of output 2t+1 is the mirror
+// image of C (g(g(j)^1) = j^1), so g(b^1)^1 is the predecessor of b on C: one
+// chain follows C forwards, the other backwards, their gathers overlap, and
+// they stop where they meet.  p_even / p_odd = P[2t] / P[2t+1], which the
+// caller holds already, start the two chains.
 template <bool PACKED>
-__device__ __forceinline__ uint32_t colour_of(const void *S, const uint32_t *Q, const uint32_t *cb,
-                                              uint32_t t, uint32_t base, bool owned, uint32_t code,
-                                              uint32_t p_odd, uint32_t rulers, int m, uint32_t mmask,
-                                              uint32_t cap, uint32_t *gate) {
-    if (owned) {
-        const uint32_t rho = code >> 1;
-        const uint32_t rr = rho < rulers ? rho : 0u;
-        return ((__ldg(cb + (rr >> 5)) >> (rr & 31u)) ^ code) & 1u;
-    }
-    // loop without ruler: walk the g-cycle of output 2t (p_odd = P[2t+1], which
-    // the caller holds already, starts the first hop)
+__device__ __forceinline__ uint32_t loop_colour(const void *S, const uint32_t *Q, uint32_t t, uint32_t base,
+                                                uint32_t p_even, uint32_t p_odd, int m, uint32_t mmask,
+                                                uint32_t cap, uint32_t *gate) {
     const uint32_t j0 = 2u * t;
-    uint32_t j = j0, mn = j0, hops = 0, p = p_odd;
+    uint32_t f = j0, bk = j0, mn = j0, hops = 0;
+    uint32_t pf = p_odd;                 // P[f ^ 1]
+    uint32_t pb = p_even;                // P[bk]
     for (;;) {
-        j = base + (__ldg(Q + base + (p ^ 1u)) & mmask);
-        if (j == j0) break;
+        const uint32_t qf = __ldg(Q + base + (pf ^ 1u)) & mmask;        // g(f)
+        const uint32_t qb = __ldg(Q + base + (pb ^ 1u)) & mmask;        // g(bk ^ 1)
+        f = base + qf;
+        if (f == bk) break;                                             // forwards reached the part walked backwards
+        mn = min(mn, f);
+        bk = (base + qb) ^ 1u;
+        if (bk == f) break;                                             // both ends on the same output
+        mn = min(mn, bk);
         if (++hops > cap) {
             *gate = 1u;
             break;
         }
         if ((hops & 63u) == 0u && gate_raised(gate)) break;
-        mn = min(mn, j);
-        p = rec_p<PACKED>(S, j ^ 1u, m);
+        pf = rec_p<PACKED>(S, f ^ 1u, m);
+        pb = rec_p<PACKED>(S, bk, m);
     }
     return mn & 1u;
 }
 
-// Both switches of a thread on loops without ruler (the rule for inputs such as
-// the identity, a bit reversal or a transpose, whose loops have one or two
-// switches): the two cycles are walked side by side, so that their gathers
-// overlap.  p0 / p1 = P[2t+1] / P[2t+3].
-template <bool PACKED>
-__device__ __forceinline__ void colour_two_walks(const void *S, const uint32_t *Q, uint32_t t, uint32_t base,
-                                                 uint32_t p0, uint32_t p1, int m, uint32_t mmask,
-                                                 uint32_t cap, uint32_t *gate, uint32_t &c0, uint32_t &c1) {
-    const uint32_t ja = 2u * t, jb = ja + 2u;
-    uint32_t j0 = ja, j1 = jb, mn0 = ja, mn1 = jb, hops = 0;
-    bool run0 = true, run1 = true;
-    while (run0 || run1) {
-        uint32_t q0 = 0, q1 = 0;
-        if (run0) q0 = __ldg(Q + base + (p0 ^ 1u));
-        if (run1) q1 = __ldg(Q + base + (p1 ^ 1u));
-        if (run0) { j0 = base + (q0 & mmask); run0 = j0 != ja; }
-        if (run1) { j1 = base + (q1 & mmask); run1 = j1 != jb; }
-        if (!(run0 || run1)) break;
-        if (++hops > cap) {
-            *gate = 1u;
-            break;
-        }
-        if ((hops & 63u) == 0u && gate_raised(gate)) break;
-        if (run0) { mn0 = min(mn0, j0); p0 = rec_p<PACKED>(S, j0 ^ 1u, m); }
-        if (run1) { mn1 = min(mn1, j1); p1 = rec_p<PACKED>(S, j1 ^ 1u, m); }
-    }
-    c0 = mn0 & 1u;
-    c1 = mn1 & 1u;
+// colour of output 2t from the owner of switch t
+__device__ __forceinline__ uint32_t owner_colour(const uint32_t *cb, uint32_t code, uint32_t rulers) {
+    const uint32_t rho = (code >> 1) < rulers ? code >> 1 : 0u;
+    return ((__ldg(cb + (rho >> 5)) >> (rho & 31u)) ^ code) & 1u;
 }
 
 // Step 5 + output side of the level's switches + the next level's records
@@ -500,17 +481,11 @@ k_colour(const void *__restrict__ S, const uint32_t *__restrict__ Q,
             px0 = r0.x & mmask; py0 = r0.y & mmask; code0 = r0.z; own0 = code0 != none;
             px1 = r1.x & mmask; py1 = r1.y & mmask; code1 = r1.z; own1 = code1 != none;
         }
-        uint32_t c0, c1;
-        if (own0 && own1) {                                     // all but the switches of loops without ruler
-            const uint32_t a = (code0 >> 1) < rulers ? code0 >> 1 : 0u, b = (code1 >> 1) < rulers ? code1 >> 1 : 0u;
-            c0 = ((__ldg(cb + (a >> 5)) >> (a & 31u)) ^ code0) & 1u;
-            c1 = ((__ldg(cb + (b >> 5)) >> (b & 31u)) ^ code1) & 1u;
-        } else if (!own0 && !own1) {
-            colour_two_walks<PACKED>(S, Q, t, base, py0, py1, m, mmask, cap, gate, c0, c1);
-        } else {
-            c0 = colour_of<PACKED>(S, Q, cb, t, base, own0, code0, py0, rulers, m, mmask, cap, gate);
-            c1 = colour_of<PACKED>(S, Q, cb, t + 1, base, own1, code1, py1, rulers, m, mmask, cap, gate);
-        }
+        // all but the switches of loops without ruler are owned
+        const uint32_t c0 = own0 ? owner_colour(cb, code0, rulers)
+                                 : loop_colour<PACKED>(S, Q, t, base, px0, py0, m, mmask, cap, gate);
+        const uint32_t c1 = own1 ? owner_colour(cb, code1, rulers)
+                                 : loop_colour<PACKED>(S, Q, t + 1u, base, px1, py1, m, mmask, cap, gate);
         // a warp covers 64 switches: two words of the output-side stage
         store_stage_bits64(L.bits + L.word32(out_stage, (t - 2u * (threadIdx.x & 31u)) >> 5), c0, c1);
         const uint32_t r = (base >> 1) + (((t - (base >> 1)) >> 1));   // record of the upper half
