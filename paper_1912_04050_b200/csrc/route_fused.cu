@@ -270,14 +270,20 @@ k_route_fused(const uint32_t *__restrict__ P, int records, uint32_t *__restrict_
                     if (code != kNone16) {
                         c = ((list[code >> 1] >> 16) ^ code) & 1u;
                     } else {
-                        // no owner: walk the g-cycle of output 2t (at most S/2 outputs)
+                        // no owner: walk the g-cycle of output 2t (at most S/2 outputs) from
+                        // both ends; g(b ^ 1) ^ 1 is the predecessor of b on the cycle (the
+                        // cycle of 2t+1 is its mirror image), and the two chains overlap
                         const uint32_t j0 = 2u * uint32_t(t), sb = j0 & ~smask;
-                        uint32_t j = j0, mn = j0;
+                        uint32_t f = j0, bk = j0, mn = j0;
                         for (uint32_t hops = 0; hops < S; ++hops) {
-                            const uint32_t p = Pcur[j ^ 1u] & smask;
-                            j = sb + (Q[sb + (p ^ 1u)] & smask);
-                            if (j == j0) break;
-                            mn = min(mn, j);
+                            const uint32_t pf = Pcur[f ^ 1u] & smask, pb = Pcur[bk] & smask;
+                            const uint32_t qf = Q[sb + (pf ^ 1u)] & smask, qb = Q[sb + (pb ^ 1u)] & smask;
+                            f = sb + qf;
+                            if (f == bk) break;
+                            mn = min(mn, f);
+                            bk = (sb + qb) ^ 1u;
+                            if (bk == f) break;
+                            mn = min(mn, bk);
                         }
                         c = mn & 1u;
                     }
