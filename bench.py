@@ -65,7 +65,7 @@ def algorithmic_bytes_per_element(kind: str, ebytes: int, kappa: int) -> float:
         "colour": 2.0 + 4.0 + 1.0 / 16.0,
         "combine": (16.0 + 16.0 + 8.0) / k, "list_walk": 20.0 / k, "list_label": 16.0 / k / 16.0,
         "list_resolve": 24.0 / k,
-        "fused": 4.0 + (2 * 13 - 1) / 16.0,
+        "fused": 4.0 + (2 * 15 - 1) / 16.0,
     }[kind]
 
 
