@@ -171,7 +171,7 @@ constexpr int kPairGroupLog2 = kListKappa;          // pairs per ruler pair (log
 
 __global__ void __launch_bounds__(kWalkThreads)
 k_list_walk_pairs(const ulonglong2 *__restrict__ W2p, uint32_t *__restrict__ owner, uint4 *__restrict__ rec,
-                  uint32_t rulers, uint32_t pmask, uint32_t salt, uint32_t cap, uint32_t *__restrict__ gate) {
+                  uint32_t rulers, uint32_t pairs, uint32_t salt, uint32_t cap, uint32_t *__restrict__ gate) {
     const uint32_t sigma = blockIdx.x * kWalkThreads + threadIdx.x;
     if (sigma >= rulers) return;
     constexpr uint32_t kmask = (1u << kPairGroupLog2) - 1u;
@@ -182,7 +182,8 @@ k_list_walk_pairs(const ulonglong2 *__restrict__ W2p, uint32_t *__restrict__ own
     unsigned long long own = side0 ? w.y : w.x;
     uint32_t fwd = uint32_t(own >> 32), part = kUnowned, peer = sigma ^ 1u, hops = 0;
     for (;;) {
-        const uint32_t e = uint32_t(own), q = (e >> 1) & pmask, side = e & 1u, g = q >> kPairGroupLog2;
+        // (a batch need not be a power of two: an index a raised gate left undefined is clamped, not masked)
+        const uint32_t e = uint32_t(own), q = (e >> 1) < pairs ? (e >> 1) : 0u, side = e & 1u, g = q >> kPairGroupLog2;
         if ((q & kmask) == ruler_slot(g, salt, kmask)) {           // reached the next ruler pair
             peer = (2u * g + side) ^ 1u;
             break;
@@ -216,10 +217,10 @@ k_list_walk_pairs(const ulonglong2 *__restrict__ W2p, uint32_t *__restrict__ own
 // needed afterwards: with `cb` one bit per word goes there, so that the colouring
 // kernel gathers from an array 64 times smaller than the list (it stays in
 // L1/L2 next to the streaming traffic); without, the words take their minima.
-__device__ __forceinline__ uint32_t list_cycle_min(const unsigned long long *W, uint32_t e0, uint32_t wmask,
+__device__ __forceinline__ uint32_t list_cycle_min(const unsigned long long *W, uint32_t e0, uint32_t words,
                                                    uint32_t cap, uint32_t *gate) {
     unsigned long long v = __ldcg(W + e0);
-    uint32_t mn = uint32_t(v >> 32), e = uint32_t(v) & wmask, hops = 0;
+    uint32_t mn = uint32_t(v >> 32), e = uint32_t(v) < words ? uint32_t(v) : 0u, hops = 0;
     while (e != e0) {
         if (++hops > cap) {
             *gate = 1u;
@@ -227,14 +228,14 @@ __device__ __forceinline__ uint32_t list_cycle_min(const unsigned long long *W, 
         }
         v = __ldcg(W + e);
         mn = min(mn, uint32_t(v >> 32));       // words rewritten meanwhile hold the minimum of this same cycle
-        e = uint32_t(v) & wmask;
+        e = uint32_t(v) < words ? uint32_t(v) : 0u;
     }
     return mn;
 }
 
 __global__ void __launch_bounds__(kThreads)
 k_list_resolve_pairs(unsigned long long *__restrict__ W, uint32_t *__restrict__ owner,
-                     const unsigned long long *__restrict__ W2, uint32_t pairs, uint32_t wmask,
+                     const unsigned long long *__restrict__ W2, uint32_t pairs, uint32_t words,
                      uint32_t cap, uint32_t *__restrict__ gate, uint32_t *__restrict__ cb) {
     const uint32_t q = blockIdx.x * kThreads + threadIdx.x;       // pairs is a multiple of 32
     if (q >= pairs) return;
@@ -247,8 +248,8 @@ k_list_resolve_pairs(unsigned long long *__restrict__ W, uint32_t *__restrict__ 
             mn1 = (code & 1u) ? a : b;
             owner[q] = kUnowned;
         } else {
-            mn0 = list_cycle_min(W, 2u * q, wmask, cap, gate);
-            mn1 = list_cycle_min(W, 2u * q + 1u, wmask, cap, gate);
+            mn0 = list_cycle_min(W, 2u * q, words, cap, gate);
+            mn1 = list_cycle_min(W, 2u * q + 1u, words, cap, gate);
         }
         ulonglong2 *Wp = reinterpret_cast<ulonglong2 *>(W) + q;
         ulonglong2 w = *Wp;
@@ -262,7 +263,7 @@ k_list_resolve_pairs(unsigned long long *__restrict__ W, uint32_t *__restrict__ 
         bit0 = (uint32_t(__ldcg(W2 + (code >> 1)) >> 32) ^ code) & 1u;
         owner[q] = kUnowned;
     } else {
-        bit0 = list_cycle_min(W, 2u * q, wmask, cap, gate) & 1u;
+        bit0 = list_cycle_min(W, 2u * q, words, cap, gate) & 1u;
     }
     // a warp covers 64 words: two words of cb
     store_stage_bits64(cb + ((q - (threadIdx.x & 31u)) >> 4), bit0, bit0 ^ 1u);
@@ -597,7 +598,7 @@ int sampled_label(void *S, bool packed, const uint32_t *Q, void *Sn, bool next_p
         {
             ProfileScope ps(kListWalk, s);
             k_list_walk_pairs<<<(next + kWalkThreads - 1) / kWalkThreads, kWalkThreads, 0, s>>>(
-                reinterpret_cast<const ulonglong2 *>(sc.list[d]), sc.owner[d], sc.rec, next, (count >> 1) - 1u,
+                reinterpret_cast<const ulonglong2 *>(sc.list[d]), sc.owner[d], sc.rec, next, count >> 1,
                 salt * 7u + uint32_t(d) + 1u, cap, gate);
             int rc = launch_status();
             if (rc) return rc;
@@ -625,7 +626,7 @@ int sampled_label(void *S, bool packed, const uint32_t *Q, void *Sn, bool next_p
         ProfileScope ps(kListResolve, s);
         const uint32_t c = R >> (kListKappa * d);
         k_list_resolve_pairs<<<(c / 2 + kThreads - 1) / kThreads, kThreads, 0, s>>>(
-            sc.list[d], sc.owner[d], sc.list[d + 1], c / 2, c - 1u, cap, gate, d == 0 ? cb : nullptr);
+            sc.list[d], sc.owner[d], sc.list[d + 1], c / 2, c, cap, gate, d == 0 ? cb : nullptr);
         int rc = launch_status();
         if (rc) return rc;
     }

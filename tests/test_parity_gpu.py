@@ -120,6 +120,20 @@ def test_route_walks_that_give_up_fall_back_to_full_pointer_jumping(cap, labelli
         assert np.array_equal(gpu_route(perm, n), oracle.route(perm, n))
 
 
+@pytest.mark.parametrize("kappa,cap", [(None, None), (2, None), (4, None), (None, 12)])
+@pytest.mark.parametrize("n,batch", [(18, 3), (19, 3), (20, 5), (19, 7)])
+def test_route_batch_not_a_power_of_two_with_resampled_lists(n, batch, kappa, cap, labelling_options):
+    """Blocks of 2^(15 + kappa) outputs and more have their contracted list sampled
+    again; the list of a batch that is not a power of two is not one either, so
+    every list index has to be bounded by the list's length, not by a mask."""
+    if kappa is not None:
+        binding.benes_set_option(binding.OPT_SAMPLE_LOG2K, kappa)
+    if cap is not None:
+        binding.benes_set_option(binding.OPT_WALK_CAP, cap)
+    perm = inputs.random_perm_batch(n, batch, seed0=31 * n + batch)
+    assert np.array_equal(gpu_route(perm, n), oracle.route(perm, n))
+
+
 @pytest.mark.parametrize("n,batch", [(22, 1), (16, 64), (17, 64), (23, 1), (16, 65)])
 def test_route_bucketed_inverse(n, batch):
     """batch * N >= 2^22 in whole multiples of 2^18 takes the two-pass inverse at
