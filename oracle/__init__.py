@@ -41,7 +41,12 @@ def _load():
         lib.oracle_route_batch.argtypes = [u32p, ctypes.c_int, ctypes.c_int, u32p]
         lib.oracle_apply_batch.argtypes = [u32p, ctypes.c_void_p, ctypes.c_void_p,
                                            ctypes.c_int, ctypes.c_int, ctypes.c_int]
-        for f in (lib.oracle_route_trace, lib.oracle_route_batch, lib.oracle_apply_batch):
+        lib.oracle_route_part.argtypes = [u32p, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_size_t,
+                                          ctypes.c_size_t, u32p, u32p]
+        lib.oracle_apply_part.argtypes = [u32p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int,
+                                          ctypes.c_int, ctypes.c_int, ctypes.c_size_t, ctypes.c_size_t]
+        for f in (lib.oracle_route_trace, lib.oracle_route_batch, lib.oracle_apply_batch,
+                  lib.oracle_route_part, lib.oracle_apply_part):
             f.restype = ctypes.c_int
         _lib = lib
     return _lib
@@ -99,6 +104,79 @@ def apply(bits: np.ndarray, x: np.ndarray, log2n: int) -> np.ndarray:
                                     x.dtype.itemsize, log2n, batch)
     if rc != 0:
         raise RuntimeError("oracle_apply_batch failed (%d)" % rc)
+    return out.reshape(x.shape)
+
+
+def _split_level(log2n: int, threads: int) -> int:
+    """First level whose sub-networks are handed to `threads` host threads: the
+    smallest level with at least `threads` sub-networks, each of 64 outputs or more."""
+    level = 0
+    while (1 << level) < threads and log2n - (level + 1) >= 6:
+        level += 1
+    return level
+
+
+def _run_parts(threads: int, jobs):
+    from concurrent.futures import ThreadPoolExecutor
+    with ThreadPoolExecutor(max_workers=threads) as pool:      # ctypes releases the GIL
+        for rc in pool.map(lambda job: job(), jobs):
+            if rc != 0:
+                raise RuntimeError("oracle part failed (%d)" % rc)
+
+
+def route_parallel(perm: np.ndarray, log2n: int, threads: int) -> np.ndarray:
+    """Same result as ``route``.  A batch: permutations are spread over `threads` host
+    threads.  One permutation: the levels above ``_split_level`` run on one thread, the
+    independent sub-networks below them on `threads` threads (same C routine, by range)."""
+    perm = np.ascontiguousarray(perm, dtype=np.uint32)
+    n, N, lib = log2n, 1 << log2n, _load()
+    p2 = perm.reshape(-1, N)
+    bits = np.zeros((p2.shape[0], 2 * n - 1, stage_words(n)), dtype=np.uint32)
+    if p2.shape[0] > 1:
+        step = -(-p2.shape[0] // threads)
+        _run_parts(threads, [
+            (lambda a=a: lib.oracle_route_batch(_u32(p2[a:a + step]), n, len(p2[a:a + step]), _u32(bits[a:a + step])))
+            for a in range(0, p2.shape[0], step)])
+    else:
+        split = _split_level(n, threads)
+        mid = np.empty(N, dtype=np.uint32)
+        rc = lib.oracle_route_part(_u32(p2[0]), n, 0, split, 0, N, _u32(bits[0]), _u32(mid))
+        if rc != 0:
+            raise RuntimeError("oracle_route_part failed (%d)" % rc)
+        M = N >> split
+        _run_parts(threads, [
+            (lambda lo=lo: lib.oracle_route_part(_u32(mid), n, split, n, lo, lo + M, _u32(bits[0]), None))
+            for lo in range(0, N, M)])
+    return bits[0] if perm.ndim == 1 else bits
+
+
+def apply_parallel(bits: np.ndarray, x: np.ndarray, log2n: int, threads: int) -> np.ndarray:
+    """Same result as ``apply``; the stages strictly inside ``_split_level`` form
+    independent sub-networks and run on `threads` host threads."""
+    n, N, lib = log2n, 1 << log2n, _load()
+    x = np.ascontiguousarray(x)
+    bits = np.ascontiguousarray(bits, dtype=np.uint32)
+    x2 = x.reshape(-1, N)
+    batch, e = x2.shape[0], x.dtype.itemsize
+    b2 = bits.reshape(batch, 2 * n - 1, stage_words(n))
+    out = x2.copy()
+    tmp = np.empty_like(out)
+    if batch > 1:
+        _run_parts(threads, [
+            (lambda b=b: lib.oracle_apply_part(_u32(b2[b]), out[b].ctypes.data, tmp[b].ctypes.data, e, n,
+                                               0, 2 * n - 1, 0, N))
+            for b in range(batch)])
+    else:
+        split = _split_level(n, threads)
+        M = N >> split
+        args = (_u32(b2[0]), out[0].ctypes.data, tmp[0].ctypes.data, e, n)
+        if lib.oracle_apply_part(*args, 0, split, 0, N) != 0:
+            raise RuntimeError("oracle_apply_part failed")
+        _run_parts(threads, [
+            (lambda lo=lo: lib.oracle_apply_part(*args, split, 2 * n - 1 - split, lo, lo + M))
+            for lo in range(0, N, M)])
+        if lib.oracle_apply_part(*args, 2 * n - 1 - split, 2 * n - 1, 0, N) != 0:
+            raise RuntimeError("oracle_apply_part failed")
     return out.reshape(x.shape)
 
 

@@ -186,3 +186,90 @@ int oracle_apply_batch(const uint32_t *bits, const void *in, void *out, int elem
     }
     return 0;
 }
+
+/*
+ * The two functions below run the SAME per-block routine and the SAME per-switch
+ * loop as oracle_route_trace / oracle_apply, restricted to a range of the flat
+ * array, so that a caller can hand independent sub-networks to several host
+ * threads (the benchmark's all-core figure: top levels on one thread, the
+ * sub-networks below them in parallel).  They add no arithmetic of their own;
+ * tests/test_oracle_pins.py checks that any split into parts reproduces
+ * oracle_route and oracle_apply word for word.
+ */
+
+/*
+ * Levels first .. stop-1 (stop <= n) of the sub-networks that occupy the flat
+ * range [lo, hi) at level `first` (lo and hi multiples of N >> first).
+ *   P_first : the flat level-`first` array of block-local sub-permutations
+ *             (N entries; only [lo, hi) is read)
+ *   bits    : the permutation's whole (2n-1) x W array, NOT cleared here; only
+ *             switches [lo/2, hi/2) of stages first..stop-1 and their mirror
+ *             stages are set.  Concurrent callers need ranges whose switches do
+ *             not share a 32-bit word: (hi - lo) a multiple of 64.
+ *   P_stop  : if not NULL and stop < n, receives the level-`stop` array on [lo, hi)
+ */
+int oracle_route_part(const uint32_t *P_first, int n, int first, int stop, size_t lo, size_t hi,
+                      uint32_t *bits, uint32_t *P_stop) {
+    if (!P_first || !bits || n < 1 || n > 30 || first < 0 || stop > n || first > stop) return -1;
+    size_t N = (size_t)1 << n, W = stage_words(n), M0 = N >> first, len = hi - lo;
+    if (lo > hi || hi > N || lo % M0 || hi % M0) return -1;
+    if (len == 0) return 0;
+    uint32_t *P = malloc(len * 4), *Pn = malloc(len * 4), *inv = malloc(len * 4);
+    uint8_t *colour = malloc(len);
+    if (!P || !Pn || !inv || !colour) { free(P); free(Pn); free(inv); free(colour); return -1; }
+    memcpy(P, P_first + lo, len * 4);
+    for (int l = first; l < stop; ++l) {
+        size_t M = N >> l;
+        if (M == 2) {
+            for (size_t b = 0; b < len / 2; ++b) set_bit(bits + (size_t)(n - 1) * W, lo / 2 + b, P[2 * b]);
+            break;
+        }
+        for (size_t base = 0; base < len; base += M)
+            route_block(P + base, M, inv, colour + base, bits + (size_t)l * W,
+                        bits + (size_t)(2 * n - 2 - l) * W, (lo + base) / 2, Pn + base);
+        uint32_t *t = P; P = Pn; Pn = t;
+    }
+    if (P_stop && stop < n) memcpy(P_stop + lo, P, len * 4);
+    free(P); free(Pn); free(inv); free(colour);
+    return 0;
+}
+
+/*
+ * Stages st_first .. st_stop-1 of oracle_apply on the positions [lo, hi), which
+ * must consist of whole blocks of every stage in that range.  x and tmp are
+ * N-element buffers; the stages ping-pong between them inside [lo, hi) and the
+ * result is left in x.
+ */
+int oracle_apply_part(const uint32_t *bits, void *xv, void *tmpv, int elem_bytes, int n,
+                      int st_first, int st_stop, size_t lo, size_t hi) {
+    if (!bits || !xv || !tmpv || n < 1 || n > 30 || elem_bytes < 1) return -1;
+    if (st_first < 0 || st_stop > 2 * n - 1 || st_first > st_stop) return -1;
+    size_t N = (size_t)1 << n, W = stage_words(n), e = (size_t)elem_bytes;
+    if (lo > hi || hi > N) return -1;
+    unsigned char *x = xv, *y = tmpv;
+    for (int st = st_first; st < st_stop; ++st) {
+        const uint32_t *stage = bits + (size_t)st * W;
+        int l = st <= n - 1 ? st : 2 * n - 2 - st;
+        size_t M = N >> l, H = M / 2;
+        if (lo % M || hi % M) return -1;
+        for (size_t base = lo; base < hi; base += M) {
+            for (size_t s = 0; s < H; ++s) {
+                uint32_t cross = get_bit(stage, base / 2 + s);
+                size_t a, b, ya, yb;
+                if (st < n - 1) {
+                    a = base + 2 * s; b = a + 1; ya = base + s; yb = base + H + s;
+                } else if (st == n - 1) {
+                    a = base; b = base + 1; ya = a; yb = b;
+                } else {
+                    a = base + s; b = base + H + s; ya = base + 2 * s; yb = ya + 1;
+                }
+                if (cross) { size_t t = a; a = b; b = t; }
+                memcpy(y + ya * e, x + a * e, e);
+                memcpy(y + yb * e, x + b * e, e);
+            }
+        }
+        unsigned char *t = x; x = y; y = t;
+    }
+    if (x != (unsigned char *)xv) memcpy((unsigned char *)xv + lo * e, x + lo * e, (hi - lo) * e);
+    return 0;
+}

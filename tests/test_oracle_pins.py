@@ -243,10 +243,8 @@ def test_all_settings_n8_canonical_is_unique_and_is_the_oracle():
     assert len(uniq) == 40320                             # rearrangeable: every permutation occurs
     order = np.argsort(key, kind="stable")
     skey = key[order]
-    rng = np.random.default_rng(8)
     perms = all_perms(N)
-    picks = rng.choice(len(perms), size=250, replace=False)
-    for perm in perms[picks]:
+    for perm in perms:                                    # every one of the 40320
         k = int((perm.astype(np.int64) * (N ** np.arange(N, dtype=np.int64))).sum())
         lo, hi = np.searchsorted(skey, k, "left"), np.searchsorted(skey, k, "right")
         members = sw[order[lo:hi]]
@@ -389,3 +387,73 @@ def test_butterfly_form_random(n):
     # identity: nothing crossed in either form
     ident = inputs.identity_perm(n)
     assert not oracle.export_butterfly(oracle.route(ident, n), n).any()
+
+
+def _pack_rows(rows):
+    """list of 0/1 lists (switch 0 first) -> (len, 1) uint32 words"""
+    return np.array([[sum(b << i for i, b in enumerate(r))] for r in rows], dtype=np.uint32)
+
+
+def test_butterfly_bit_order_hand_traced_rows():
+    """tests/golden/butterfly_rows_n8.txt: the order of the bits inside a row, traced by hand."""
+    n = 3
+    with open(os.path.join(GOLDEN, "butterfly_rows_n8.txt")) as f:
+        lines = [ln for ln in f if ln.strip() and not ln.startswith("#")]
+    assert len(lines) == 2
+    for ln in lines:
+        rec, inplace = ([[int(v) for v in row.split()] for row in side.split("|")] for side in ln.split(";"))
+        assert np.array_equal(oracle.export_butterfly(_pack_rows(rec), n), _pack_rows(inplace))
+
+
+def _bitrev(v, width):
+    r = 0
+    for i in range(width):
+        r |= ((v >> i) & 1) << (width - 1 - i)
+    return r
+
+
+@pytest.mark.parametrize("n", [2, 3, 4, 6, 9, 11])
+def test_butterfly_bit_order_closed_form(n):
+    """Block b of level l (its bits are the up/down choices of levels 0..l-1, first choice on
+    top) keeps choice k in bit k of the in-place position, and position r of the block sits
+    above them: in-place position = r << l | reverse_l(b).  So recursive switch w = (b, s) of
+    level l is in-place switch s << l | reverse_l(b), on both sides of the network."""
+    rng = np.random.default_rng(n)
+    N, W = 1 << n, max(1, (1 << n) // 64)
+    bits = rng.integers(0, 2, size=(2 * n - 1, N // 2), dtype=np.uint8)
+    want = np.zeros_like(bits)
+    for r in range(2 * n - 1):
+        l = r if r <= n - 1 else 2 * n - 2 - r
+        per_block = 1 << (n - l - 1)
+        for w in range(N // 2):
+            b, s = w // per_block, w % per_block
+            want[r, (s << l) | _bitrev(b, l)] = bits[r, w]
+
+    def pack(a):
+        full = np.zeros((2 * n - 1, W * 32), dtype=np.uint8)
+        full[:, :N // 2] = a
+        return np.packbits(full, axis=1, bitorder="little").view(np.uint32).reshape(2 * n - 1, W)
+
+    assert np.array_equal(oracle.export_butterfly(pack(bits), n), pack(want))
+
+
+# ---- range-restricted entry points (the benchmark's all-core leg) ------------------------
+@pytest.mark.parametrize("n", [1, 2, 5, 6, 7, 8, 11, 15])
+@pytest.mark.parametrize("threads", [1, 2, 3, 16])
+def test_parts_reproduce_the_whole(n, threads):
+    """Top levels on one thread, the sub-networks below on several: same words, same payload."""
+    perm = inputs.random_perm(n, 300 + n)
+    bits = oracle.route(perm, n)
+    assert np.array_equal(oracle.route_parallel(perm, n, threads), bits)
+    x = inputs.payload_u64(1 << n, n)
+    out = oracle.apply_parallel(bits, x, n, threads)
+    assert np.array_equal(out, oracle.apply(bits, x, n))
+    assert np.array_equal(out, x[perm])
+
+
+def test_parts_batched():
+    perm = inputs.random_perm_batch(7, 21, seed0=3)
+    bits = oracle.route(perm, 7)
+    assert np.array_equal(oracle.route_parallel(perm, 7, 4), bits)
+    x = np.arange(21 << 7, dtype=np.uint32).reshape(21, -1)
+    assert np.array_equal(oracle.apply_parallel(bits, x, 7, 4), oracle.apply(bits, x, 7))
