@@ -4,17 +4,22 @@
 One "step" = one pass of the whole path over one synthetic input: benes_route
 (all levels) followed by benes_apply_ex of a payload through the 2n-1 stages.
 Default workload: a single uniform random permutation of N = 2^26 (uint32,
-Fisher-Yates seed 2) with a 2^26-element uint64 payload.  With --gpus N every
-rank routes its own permutation (seed 2 + rank): batch replicas, no collective
-on the data path, weak scaling.
+Fisher-Yates seed 2) with a 2^26-element uint64 payload.
+
+--gpus N: one process per GPU, every rank routes its own permutation (seed
+2 + rank): batch replicas, no collective on the data path, weak scaling.  Under
+torchrun the ranks come from the environment; started plainly with --gpus N > 1
+this script starts the N ranks itself.
 
 Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
 """
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
+import socket
 import statistics
 import subprocess
 import sys
@@ -33,17 +38,24 @@ WORKLOADS = {
     "c4": (26, 1, 8, 2, "C4: 1 x N=2^26 uniform random permutation (Fisher-Yates seed 2), route + uint64 payload apply"),
     "c3": (20, 1, 4, 1, "C3: 1 x N=2^20 uniform random permutation (seed 1), route + fp32 payload apply"),
     "c2": (8, 16384, 4, 0, "C2: 16384 x N=2^8 uniform random permutations (seeds 0..16383), route + uint32 payload apply"),
+    "c1": (10, 1, 4, 0, "C1: 1 x N=2^10 uniform random permutation (seed 0), route + uint32 identity payload apply"),
     "r25": (25, 1, 8, 2, "profiling case: 1 x N=2^25 uniform random permutation (seed 2), route + uint64 payload apply"),
+    "r22": (22, 1, 8, 2, "profiling case: 1 x N=2^22 uniform random permutation (seed 2), route + uint64 payload apply"),
     "c5s": (24, 1, 4, 3, "C5: 1 x N=2^24 Sattolo single-cycle permutation (seed 3), route + uint32 payload apply"),
     "m10": (10, 16384, 4, 0, "mid-size batch: 16384 x N=2^10 uniform random permutations, route + uint32 payload apply"),
     "m12": (12, 4096, 4, 0, "mid-size batch: 4096 x N=2^12 uniform random permutations, route + uint32 payload apply"),
     "m16": (16, 256, 4, 0, "mid-size batch: 256 x N=2^16 uniform random permutations, route + uint32 payload apply"),
+    "m17": (17, 128, 4, 0, "mid-size batch: 128 x N=2^17 uniform random permutations, route + uint32 payload apply"),
     "c5i": (24, 1, 4, 0, "C5: 1 x N=2^24 identity, route + uint32 payload apply"),
     "c5h": (24, 1, 4, 0, "C5: 1 x N=2^24 cyclic shift by 1, route + uint32 payload apply"),
     "c5b": (24, 1, 4, 0, "C5: 1 x N=2^24 bit reversal, route + uint32 payload apply"),
     "c5t": (24, 1, 4, 0, "C5: 1 x N=2^24 index map of a 4096x4096 transpose, route + uint32 payload apply"),
 }
 STRUCTURED = {"c5i": "identity", "c5h": "shift1", "c5b": "bitrev", "c5t": "transpose"}
+L2_BYTES = 126 << 20
+# workloads whose summary rides along in the default (C4) line
+SIDE_WORKLOADS = ("c3", "c2")
+
 
 def algorithmic_bytes_per_element(kind: str, ebytes: int, kappa: int) -> float:
     """Useful bytes one launch of a kernel kind moves per permutation element."""
@@ -69,16 +81,10 @@ def algorithmic_bytes_per_element(kind: str, ebytes: int, kappa: int) -> float:
     }[kind]
 
 
-# DRAM bytes per launch per element of the dominant kernel measured with ncu
-# (dram__bytes_read.sum + dram__bytes_write.sum); see profiles/.  None until captured
-# for the kernel as it stands.
-NCU_DRAM_BYTES_PER_ELEMENT = {
-    # mean over the 10 k_walk launches of one route at N = 2^25 (profiles/k_walk_n2p25.md),
-    # scaled by the elements of a launch; the top level of a larger N moves somewhat more
-    "walk": 32.8,
-}
 FALLBACK_HBM_GBS = 6650.0
-RANDOM_GATHER_PEAK_G = 64.7
+# which source file holds the kernels of a profile kind (its hash guards the stored ncu counters)
+KIND_SOURCE = {"walk": "route_sampled.cu", "colour": "route_sampled.cu", "fused": "route_fused.cu",
+               "split": "route_levels.cu", "inverse": "route_levels.cu", "apply_fused": "apply_fused.cu"}
 
 
 def measured_peaks():
@@ -88,6 +94,31 @@ def measured_peaks():
             return float(json.load(f)["hbm_gbs"]), "measured"
     except Exception:
         return FALLBACK_HBM_GBS, "fallback"
+
+
+def source_hash(fname: str) -> str:
+    with open(os.path.join(ROOT, "paper_1912_04050_b200", "csrc", fname), "rb") as f:
+        return hashlib.sha256(f.read()).hexdigest()[:16]
+
+
+def stored_dram_traffic(kind: str, workload: str):
+    """DRAM bytes per launch (read + write) of one kernel kind on one workload, from the
+    ncu counters kept as text beside the other profile summaries; None if there are none,
+    or if the kernel's source file has changed since they were taken."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.txt")
+    try:
+        with open(path) as f:
+            rows = [ln.split() for ln in f if ln.strip() and not ln.startswith("#")]
+    except OSError:
+        return None
+    for row in rows:
+        rec = dict(kv.split("=", 1) for kv in row)
+        if rec.get("kind") == kind and rec.get("workload") == workload:
+            src = KIND_SOURCE.get(kind)
+            if src is None or rec.get("source_sha") != source_hash(src):
+                return None
+            return float(rec["dram_bytes_per_launch"])
+    return None
 
 
 class ClockSampler:
@@ -185,34 +216,130 @@ def make_inputs(name: str, rank: int):
     return perm.reshape(-1), x
 
 
-# --------------------------------------------------------------------------------------------
+# ---- ranks ----------------------------------------------------------------------------------
+def _free_port() -> int:
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def spawn_ranks(world: int, argv, extra_env=None) -> int:
+    """Start `world` copies of this script, one per GPU, with the rendezvous variables
+    torchrun would set (127.0.0.1, a free port).  Returns the first non-zero exit code."""
+    port = _free_port()
+    procs = []
+    for rank in range(world):
+        env = dict(os.environ, RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(world),
+                   LOCAL_WORLD_SIZE=str(world), MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        env.update(extra_env or {})
+        procs.append(subprocess.Popen([sys.executable, os.path.abspath(__file__)] + list(argv), env=env))
+    rc = 0
+    for p in procs:
+        p.wait()
+        rc = rc or p.returncode
+    return rc
+
+
+def init_ranks(args, backend: str):
+    """(rank, local_rank, world, dist or None) from the environment; checks --gpus against it."""
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world != args.gpus:
+        raise SystemExit("bench.py: --gpus %d but WORLD_SIZE=%d" % (args.gpus, world))
+    dist = None
+    if world > 1:
+        import torch
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        if backend == "nccl":
+            dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        else:
+            dist.init_process_group(backend)
+    return rank, local_rank, world, dist
+
+
+def run_rank_check(args):
+    """The rank plumbing alone, on the CPU (gloo): every rank builds its inputs, pretends to
+    need (rank + 1) ms per step, and rank 0 prints the line skeleton.  Used by the tests."""
+    rank, _, world, dist = init_ranks(args, "gloo")
+    n, batch, _, _, desc = WORKLOADS[args.workload]
+    perm, _ = make_inputs(args.workload, rank)
+    ms_step, = max_over_ranks([1.0 + rank], dist, "cpu")
+    digest = hashlib.sha256(perm.tobytes()).hexdigest()[:16]
+    digests = [None] * world
+    if dist:
+        dist.all_gather_object(digests, digest)
+    else:
+        digests = [digest]
+    if rank == 0:
+        print(json.dumps({"metric": METRIC, "value": whole_job_value(batch << n, world, ms_step), "unit": UNIT,
+                          "n_gpus": world, "ms_per_step": ms_step, "scaling": "weak",
+                          "config": {"workload": desc}, "rank_inputs": digests}), flush=True)
+    if dist:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+# ---- CPU oracle legs -------------------------------------------------------------------------
+def oracle_step(perm, x, n, threads):
+    import oracle
+    if threads > 1:
+        bits = oracle.route_parallel(perm, n, threads)
+        return oracle.apply_parallel(bits, x, n, threads)
+    bits = oracle.route(perm, n)
+    return oracle.apply(bits, x, n)
+
+
+def oracle_inputs(name: str, n: int, batch: int):
+    import numpy as np
+    from paper_1912_04050_b200 import inputs
+    _, _, ebytes, seed, _ = WORKLOADS[name]
+    if name == "c5s":
+        perm = inputs.sattolo_perm(n, seed)
+    elif name in STRUCTURED:
+        perm = inputs.structured_perms(n)[STRUCTURED[name]]
+    else:
+        perm = inputs.random_perm_batch(n, batch, seed0=seed) if batch > 1 else inputs.random_perm(n, seed)
+    x = inputs.payload_u64(batch << n, seed) if ebytes == 8 else np.tile(inputs.identity_perm(n), batch)
+    return perm, x.reshape(batch, -1) if batch > 1 else x
+
+
 def run_reference(args):
-    """The CPU oracle as it stands, on the host cores, on a bounded sample of the workload."""
+    """The CPU oracle as it stands, one thread, on the host cores.  A step of the full C4
+    workload takes about a minute, so each step runs a bounded sample: the largest N (same
+    generator and seed) for which steps + warm-up finish within about three minutes."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    import numpy as np
-    import oracle
-    from paper_1912_04050_b200 import inputs
     n_full, batch_full, ebytes, seed, desc = WORKLOADS[args.workload]
     total = args.steps + args.warmup
-    n = min(n_full, 22 if total <= 12 else 20)
+    budget_s = 170.0
     if batch_full > 1:
-        n, batch = n_full, min(batch_full, 4096)
-        perm = inputs.random_perm_batch(n, batch, seed0=seed)
-        sample = "first %d of the %d permutations of N=2^%d" % (batch, batch_full, n)
+        n, batch = n_full, batch_full
+        perm, x = oracle_inputs(args.workload, n, batch)
+        t0 = time.perf_counter(); oracle_step(perm[:256], x[:256], n, 1); t256 = time.perf_counter() - t0
+        while batch > 256 and t256 * (batch / 256.0) * total > budget_s:
+            batch //= 2
+        perm, x = perm[:batch], x[:batch]
+        sample = "first %d of the %d permutations of N=2^%d, route + apply per step" % (batch, batch_full, n)
     else:
         batch = 1
-        perm = inputs.random_perm(n, seed)
-        sample = ("one uniform random permutation of N=2^%d (same generator and seed as the "
-                  "N=2^%d workload), route + %d-byte payload apply per step" % (n, n_full, ebytes))
-    x = inputs.payload_u64(batch << n, seed) if ebytes == 8 else np.tile(inputs.identity_perm(n), batch)
-    x = x.reshape(batch, -1)
+        n_cal = min(n_full, 20)
+        perm, x = oracle_inputs(args.workload, n_cal, 1)
+        t0 = time.perf_counter(); oracle_step(perm, x, n_cal, 1); t_cal = time.perf_counter() - t0
+        n = n_cal
+        # time per element grows slowly with N (cache misses): allow 15 % per doubling
+        while n < n_full and t_cal * (2.3 ** (n + 1 - n_cal)) * total <= budget_s:
+            n += 1
+        perm, x = oracle_inputs(args.workload, n, 1)
+        sample = ("one uniform random permutation of N=2^%d (same generator and seed as the N=2^%d "
+                  "workload; the largest size whose %d steps fit in about %d s), route + %d-byte payload "
+                  "apply per step" % (n, n_full, total, int(budget_s), ebytes))
     times = []
     for i in range(total):
         t0 = time.perf_counter()
-        bits = oracle.route(perm, n)
-        out = oracle.apply(bits, x, n)
+        out = oracle_step(perm, x, n, 1)
         dt = time.perf_counter() - t0
         if i >= args.warmup:
             times.append(dt)
@@ -224,8 +351,9 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "u32", "data": "synthetic",
-        "config": {"workload": desc, "reference_sample": sample},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "config": {"workload": desc, "reference_sample": sample, "sample_log2n": n, "sample_batch": batch},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "nproc": os.cpu_count(),
+                         "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -233,47 +361,155 @@ def run_reference(args):
 
 
 def time_cpu_baseline(name: str):
-    """Oracle on a bounded sample (about 10-30 s of single-core work)."""
+    """The oracle, once, on the benched workload itself (same generator, seed and size):
+    single thread (the oracle is sequential by definition), then on all host cores over
+    independent units only (permutations of a batch; for one permutation the sub-networks
+    below level ceil(log2 cores), the levels above them on one thread)."""
     import numpy as np
-    import oracle
-    from paper_1912_04050_b200 import inputs
-    n_full, batch_full, ebytes, seed, _ = WORKLOADS[name]
-    if batch_full > 1:
-        n, batch = n_full, batch_full
-        perm = inputs.random_perm_batch(n, batch, seed0=seed)
-        sample = "all %d permutations of N=2^%d, route + apply, once" % (batch, n)
-    else:
-        n, batch = min(n_full, 23), 1
-        perm = inputs.random_perm(n, seed)
-        sample = ("one uniform random permutation of N=2^%d (same generator and seed), route + "
-                  "%d-byte payload apply, once, single thread" % (n, ebytes))
-    x = inputs.payload_u64(batch << n, seed) if ebytes == 8 else np.tile(inputs.identity_perm(n), batch)
-    x = x.reshape(batch, -1)
+    n, batch, ebytes, _, _ = WORKLOADS[name]
+    perm, x = oracle_inputs(name, n, batch)
+    cores = os.cpu_count() or 1
     t0 = time.perf_counter()
-    bits = oracle.route(perm, n)
-    oracle.apply(bits, x, n)
-    dt = time.perf_counter() - t0
-    return {"value": (batch << n) / dt, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample,
-            "seconds": dt}
+    out1 = oracle_step(perm, x, n, 1)
+    dt1 = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    outp = oracle_step(perm, x, n, cores)
+    dtp = time.perf_counter() - t0
+    assert np.array_equal(out1, outp)
+    what = ("all %d permutations of N=2^%d" % (batch, n)) if batch > 1 else ("the whole N=2^%d permutation" % n)
+    return {"value": (batch << n) / dt1, "unit": UNIT, "cores": 1, "kind": "oracle", "nproc": cores,
+            "sample": "%s (same generator and seed as the GPU run), route + %d-byte payload apply, once, one thread"
+                      % (what, ebytes),
+            "seconds": dt1,
+            "all_cores": {"value": (batch << n) / dtp, "unit": UNIT, "cores": cores, "seconds": dtp,
+                          "how": ("permutations spread over the threads" if batch > 1 else
+                                  "levels above the split on one thread, the independent sub-networks "
+                                  "below it on %d threads" % cores)}}
 
 
-# --------------------------------------------------------------------------------------------
+# ---- GPU legs --------------------------------------------------------------------------------
+class GpuCase:
+    """Device-resident inputs and outputs of one workload on the current device."""
+
+    def __init__(self, name: str, rank: int, stream):
+        import numpy as np
+        import torch
+        from paper_1912_04050_b200 import binding
+        self.name, self.stream, self.binding = name, stream, binding
+        self.n, self.batch, self.ebytes, _, self.desc = WORKLOADS[name]
+        self.perm_h, self.x_h = make_inputs(name, rank)
+        self.elems = self.batch << self.n
+        self.view = {4: np.int32, 8: np.int64}[self.ebytes]
+        self.d_perm = torch.from_numpy(self.perm_h.view(np.int32)).cuda()
+        self.d_x = torch.from_numpy(self.x_h.view(self.view)).cuda()
+        self.d_bits = torch.empty(binding.benes_switch_words(self.n, self.batch), dtype=torch.int32, device="cuda")
+        self.d_out = torch.empty_like(self.d_x)
+        self.input_bytes = self.perm_h.nbytes + self.x_h.nbytes
+
+    def step(self):
+        b = self.binding
+        b.benes_route(self.d_perm, self.n, self.batch, self.d_bits, self.stream)
+        b.benes_apply_ex(self.d_bits, self.d_x, self.d_out, self.ebytes, self.n, self.batch, self.stream)
+
+    def check(self):
+        """the routed payload must equal the gather (on the device)"""
+        import torch
+        idx = self.d_perm.view(self.batch, -1).to(torch.int64) & 0xFFFFFFFF
+        ok = torch.equal(self.d_out.view(self.batch, -1), torch.gather(self.d_x.view(self.batch, -1), 1, idx))
+        assert ok, "routed payload wrong (%s)" % self.name
+
+
+class L2Flush:
+    """Writes a buffer twice the size of the L2 between timed iterations of small workloads."""
+
+    def __init__(self):
+        import torch
+        self.buf = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device="cuda")
+
+    def __call__(self):
+        self.buf.fill_(1)
+
+
+def time_steps(case: GpuCase, steps: int, flush):
+    """Per-step device times (ms).  Inputs above the L2 size run back to back inside one
+    event pair; smaller ones are timed step by step with the L2 flushed in between."""
+    import torch
+    s = case.stream
+    if flush is None:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(s)
+        for _ in range(steps):
+            case.step()
+        e1.record(s)
+        torch.cuda.synchronize()
+        return [e0.elapsed_time(e1) / steps] * steps
+    pairs = []
+    for _ in range(steps):
+        flush()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(s)
+        case.step()
+        e1.record(s)
+        pairs.append((e0, e1))
+    torch.cuda.synchronize()
+    return [a.elapsed_time(b) for a, b in pairs]
+
+
+def probe_gather(binding, table, stream):
+    """Independent random 4-byte gathers from `table` (a power-of-two number of words): G/s."""
+    import torch
+    words = table.numel()
+    log2w = words.bit_length() - 1
+    sink = torch.zeros(1, dtype=torch.int32, device="cuda")
+    gathers = min(1 << 28, max(1 << 24, 4 * words))
+    best = None
+    for i in range(6):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        binding.benes_probe_gather(table, log2w, gathers, sink, stream)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        if i >= 2:
+            ms = e0.elapsed_time(e1)
+            best = ms if best is None else min(best, ms)
+    return {"value": gathers / (best * 1e-3) / 1e9, "unit": "G gathers/s", "gathers": gathers,
+            "table_bytes": words * 4, "ms": best}
+
+
+def side_workload(name: str, rank: int, stream, flush, steps: int = 10):
+    """Short summary of another configuration (device-resident, L2 flushed between steps)."""
+    import torch
+    case = GpuCase(name, rank, stream)
+    with torch.cuda.stream(stream):
+        for _ in range(3):
+            case.step()
+        torch.cuda.synchronize()
+        case.check()
+        ms = time_steps(case, steps, flush)
+        r0, r1, r2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+        flush()
+        r0.record(stream)
+        case.binding.benes_route(case.d_perm, case.n, case.batch, case.d_bits, stream)
+        r1.record(stream)
+        case.binding.benes_apply_ex(case.d_bits, case.d_x, case.d_out, case.ebytes, case.n, case.batch, stream)
+        r2.record(stream)
+        torch.cuda.synchronize()
+    med = statistics.median(ms)
+    return {"workload": case.desc, "ms_per_step": med, "best_ms": min(ms), "steps": steps,
+            "value": case.elems / (med * 1e-3), "unit": UNIT, "l2": "flushed between steps",
+            "route_ms": r0.elapsed_time(r1), "apply_ms": r1.elapsed_time(r2)}
+
+
 def run_gpu(args):
     import numpy as np
     import torch
     from paper_1912_04050_b200 import binding
     from paper_1912_04050_b200 import build as cuda_build
 
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    rank, local_rank, world, dist = init_ranks(args, "nccl")
     torch.cuda.set_device(local_rank)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     if rank == 0:
         cuda_build.build()
     if dist:
@@ -283,19 +519,11 @@ def run_gpu(args):
         binding.benes_set_option(binding.OPT_SAMPLE_LOG2K, args.kappa)
 
     name = args.workload
-    n, batch, ebytes, seed, desc = WORKLOADS[name]
-    perm_h, x_h = make_inputs(name, rank)
-    elems = batch << n
-    view = {4: np.int32, 8: np.int64}
-    d_perm = torch.from_numpy(perm_h.view(np.int32)).cuda()
-    d_x = torch.from_numpy(x_h.view(view[ebytes])).cuda()
-    d_bits = torch.empty(binding.benes_switch_words(n, batch), dtype=torch.int32, device="cuda")
-    d_out = torch.empty_like(d_x)
     stream = torch.cuda.Stream()
-
-    def step():
-        binding.benes_route(d_perm, n, batch, d_bits, stream)
-        binding.benes_apply_ex(d_bits, d_x, d_out, ebytes, n, batch, stream)
+    case = GpuCase(name, rank, stream)
+    n, batch, ebytes, elems = case.n, case.batch, case.ebytes, case.elems
+    flush = None if case.input_bytes > L2_BYTES else L2Flush()
+    warmup = max(args.warmup, 3)
 
     def fence():
         torch.cuda.synchronize()
@@ -304,15 +532,13 @@ def run_gpu(args):
             torch.cuda.synchronize()
 
     with torch.cuda.stream(stream):
-        for _ in range(max(args.warmup, 3)):
-            step()
+        for _ in range(warmup):
+            case.step()
         fence()
-        # correctness guard: the routed payload must equal the gather (cheap, on device)
-        idx = d_perm.view(batch, -1).to(torch.int64) & 0xFFFFFFFF
-        assert torch.equal(d_out.view(batch, -1), torch.gather(d_x.view(batch, -1), 1, idx)), "routed payload wrong"
-        del idx
+        case.check()
 
-        # ---- timed region: device-resident inputs ----
+        # ---- timed region: device-resident inputs.  The library's per-kind event brackets are
+        # on (two event records per group of launches), so `value` includes their cost.
         sampler = ClockSampler(gpu_index(local_rank))
         if rank == 0:
             sampler.start()
@@ -321,15 +547,9 @@ def run_gpu(args):
         binding.benes_profile_enable(True)
         fence()
         l0 = binding.benes_launch_count()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        for _ in range(args.steps):
-            step()
-        e1.record(stream)
+        step_ms = time_steps(case, args.steps, flush)
         fence()
         launches = binding.benes_launch_count() - l0
-        ms_total = e0.elapsed_time(e1)
         binding.benes_profile_enable(False)
         kinds = {}
         for k in range(binding.PROFILE_KINDS):
@@ -342,20 +562,20 @@ def run_gpu(args):
         binding.benes_profile_reset()
         clocks = sampler.stop() if rank == 0 else None
 
-        # route-only / apply-only split (one extra untimed-for-value pass each)
+        # route-only / apply-only split (one extra pass, not part of `value`)
+        r0, r1, r2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
         r0.record(stream)
-        binding.benes_route(d_perm, n, batch, d_bits, stream)
+        binding.benes_route(case.d_perm, n, batch, case.d_bits, stream)
         r1.record(stream)
-        binding.benes_apply_ex(d_bits, d_x, d_out, ebytes, n, batch, stream)
-        e1b = torch.cuda.Event(enable_timing=True)
-        e1b.record(stream)
+        binding.benes_apply_ex(case.d_bits, case.d_x, case.d_out, ebytes, n, batch, stream)
+        r2.record(stream)
         fence()
-        route_ms, apply_ms = r0.elapsed_time(r1), r1.elapsed_time(e1b)
+        route_ms, apply_ms = r0.elapsed_time(r1), r1.elapsed_time(r2)
 
         # ---- end to end: host buffers through the C ABI, copies inside the timed region ----
-        perm_p = torch.from_numpy(perm_h.view(np.int32)).pin_memory()
-        x_p = torch.from_numpy(x_h.view(view[ebytes])).pin_memory()
-        bits_p = torch.empty(d_bits.numel(), dtype=torch.int32).pin_memory()
+        perm_p = torch.from_numpy(case.perm_h.view(np.int32)).pin_memory()
+        x_p = torch.from_numpy(case.x_h.view(case.view)).pin_memory()
+        bits_p = torch.empty(case.d_bits.numel(), dtype=torch.int32).pin_memory()
         out_p = torch.empty_like(x_p).pin_memory()
 
         def e2e_step():
@@ -373,9 +593,14 @@ def run_gpu(args):
         g1.record(stream)
         fence()
         e2e_ms = max(g0.elapsed_time(g1), 1e3 * (time.perf_counter() - t0)) / e2e_steps
-        assert torch.equal(out_p, d_out.cpu()), "end-to-end payload differs from the device-resident run"
+        assert torch.equal(out_p, case.d_out.cpu()), "end-to-end payload differs from the device-resident run"
+        del perm_p, x_p, out_p
 
-    ms_step = ms_total / args.steps
+        gather = None
+        if rank == 0 and (case.d_perm.numel() & (case.d_perm.numel() - 1)) == 0 and case.d_perm.numel() >= 1 << 20:
+            gather = probe_gather(binding, case.d_perm, stream)
+
+    ms_step = sum(step_ms) / len(step_ms)
     ms_step, e2e_ms, route_ms, apply_ms = max_over_ranks([ms_step, e2e_ms, route_ms, apply_ms], dist, "cuda")
 
     if rank == 0:
@@ -392,41 +617,45 @@ def run_gpu(args):
                 "bound": "hbm", "kernel": top,
                 "achieved": achieved, "peak": peak, "peak_source": peak_kind + " (STREAM-style copy)",
                 "unit": "GB/s", "frac": achieved / peak,
-                "traffic": (NCU_DRAM_BYTES_PER_ELEMENT[top] * elems
-                            if top in NCU_DRAM_BYTES_PER_ELEMENT else None),
+                "traffic": stored_dram_traffic(top, name),
                 "algorithmic_bytes_per_launch": bpe * elems,
                 "avg_launch_ms": per_launch_s * 1e3, "launches_timed": dom["launches"],
             }
-            if top == "walk" and per_level.get("walk"):
-                # the walk is a chain of dependent random accesses: per switch one 16-byte
-                # record and one 4-byte inverse entry (the claim hits the record's sector),
-                # i.e. one access per element.  Level 0 is the launch whose block (12 B per
-                # output) is furthest above the L2, so its accesses all go to DRAM.
+            if top == "walk" and per_level.get("walk") and gather:
+                # the walk is a chain of dependent random accesses: per switch one record and
+                # one 4-byte inverse entry (the claim hits the record's sector), i.e. one access
+                # per element.  Level 0 is the launch whose block is furthest above the L2, so
+                # its accesses all go to DRAM; the ceiling is the rate of independent random
+                # gathers from the same-sized array, measured in this run.
                 acc = float(elems) / (per_level["walk"][0] * 1e-3) / 1e9
                 roofline["random_access"] = {
                     "launch": "level 0", "ms": per_level["walk"][0],
-                    "achieved": acc, "unit": "G accesses/s", "peak": RANDOM_GATHER_PEAK_G,
-                    "peak_source": "stand-alone test on this GPU: independent random 4-byte gathers "
-                                   "from a 256 MiB array", "frac": acc / RANDOM_GATHER_PEAK_G,
-                    # the claim (a compare-and-swap on the record) counted as a third
-                    # memory operation per switch, i.e. 1.5 per element
+                    "achieved": acc, "unit": "G accesses/s", "peak": gather["value"],
+                    "peak_source": "this run: %d independent random 4-byte gathers from the %d MiB "
+                                   "permutation array (benes_probe_gather), best of 4"
+                                   % (gather["gathers"], gather["table_bytes"] >> 20),
+                    "frac": acc / gather["value"],
+                    # the claim (an atomic on the record) counted as a third memory operation
+                    # per switch, i.e. 1.5 per element
                     "achieved_with_claims": 1.5 * acc,
-                    "frac_with_claims": 1.5 * acc / RANDOM_GATHER_PEAK_G}
-        bits_bytes = d_bits.numel() * 4
+                    "frac_with_claims": 1.5 * acc / gather["value"]}
+        bits_bytes = case.d_bits.numel() * 4
         line = {
             "metric": METRIC, "value": whole_job_value(elems, world, ms_step), "unit": UNIT,
-            "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+            "n_gpus": world, "steps": args.steps, "warmup": warmup,
             "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "u32", "data": "synthetic",
-            "config": {"workload": desc, "log2n": n, "batch_per_gpu": batch, "payload_bytes": ebytes,
+            "config": {"workload": case.desc, "log2n": n, "batch_per_gpu": batch, "payload_bytes": ebytes,
                        "parallelism": "replicas x%d, no collective" % world,
-                       "l2": "inputs larger than L2 (perm %d MiB, words %d MiB)" % (elems * 4 >> 20, elems * 8 >> 20),
+                       "l2": ("inputs larger than L2 (perm %d MiB, payload %d MiB)"
+                              % (case.perm_h.nbytes >> 20, case.x_h.nbytes >> 20)) if flush is None
+                             else "L2 flushed between timed steps (a 252 MiB buffer is written)",
                        "fused_log2m": binding.benes_fused_log2m(),
                        "ruler_spacing_log2": kappa},
             "clocks": clocks,
             "e2e": {"value": world * elems / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
-                    "h2d_bytes_per_step": perm_h.nbytes + bits_bytes + x_h.nbytes,
-                    "d2h_bytes_per_step": bits_bytes + x_h.nbytes},
+                    "h2d_bytes_per_step": case.perm_h.nbytes + bits_bytes + case.x_h.nbytes,
+                    "d2h_bytes_per_step": bits_bytes + case.x_h.nbytes},
             "gpu_launches": launches,
             "roofline": roofline,
             "breakdown": {"route_ms": route_ms, "apply_ms": apply_ms,
@@ -437,6 +666,13 @@ def run_gpu(args):
                                                      if k in ("walk", "colour", "split", "list_label", "list_walk")},
                           "kernel_launches_per_step": {k: v["launches"] // args.steps for k, v in kinds.items()}},
         }
+        if gather:
+            line["gather_probe"] = gather
+        if world == 1 and name == "c4" and not args.no_side_workloads:
+            del case
+            torch.cuda.empty_cache()
+            fl = flush or L2Flush()
+            line["other_workloads"] = {w: side_workload(w, rank, stream, fl) for w in SIDE_WORKLOADS}
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = time_cpu_baseline(name)
         print(json.dumps(line), flush=True)
@@ -453,11 +689,20 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c4", choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-side-workloads", action="store_true")
     ap.add_argument("--kappa", type=int, default=None,
                     help="ruler spacing (log2) of the loop labelling; 0 = full pointer jumping")
+    ap.add_argument("--rank-check", action="store_true",
+                    help="run only the rank plumbing on the CPU (gloo); used by the tests")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started plainly: be the launcher (NCCL's own log stays on for the ranks)
+        sys.exit(spawn_ranks(args.gpus, sys.argv[1:]))
+    if args.rank_check:
+        run_rank_check(args)
     else:
         run_gpu(args)
 

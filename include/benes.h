@@ -54,6 +54,10 @@ enum {
     BENES_ERR_NOT_PERMUTATION = -4, /* benes_validate_perm only */
     BENES_ERR_TOO_LARGE = -5        /* benes_apply_static only: payload exceeds the built-in scratch */
 };
+/* There is no time-out status: no kernel of the library waits on a flag, a peer
+ * or another launch.  The only loops whose length depends on the data are the
+ * walks, and those stop after BENES_OPT_WALK_CAP hops and hand the level to the
+ * pointer-jumping kernel, whose pass count is fixed by the block size. */
 
 #define BENES_MAX_LOG2N 30
 
@@ -234,6 +238,29 @@ int benes_profile_read(int kind, unsigned long long *launches, double *milliseco
  * BENES_ERR_BADARG once index is past the last group. */
 int benes_profile_span(int index, int *kind, unsigned long long *launches, double *milliseconds);
 const char *benes_profile_kind_name(int kind);
+
+/*
+ * Batch sharding over several GPUs.  The permutations of a batch are independent,
+ * so G processes (one per GPU) each route a contiguous slice with no exchange
+ * between them: rank r of `world` takes permutations [*first, *first + *count)
+ * (slice sizes differ by at most one; *count may be 0 when world > batch) and
+ * calls benes_route / benes_apply on perm + *first * N, switch_bits +
+ * *first * (2n-1) * W and the matching payload rows.  Host-only arithmetic; no
+ * CUDA call.  A single permutation does not shard: its top levels gather over
+ * the whole array.
+ */
+int benes_shard_batch(int batch, int world, int rank, int *first, int *count);
+
+/*
+ * Measurement aid (no step of the method): `gathers` (<= 2^32) independent random
+ * 4-byte reads from table[0 .. 2^log2_words), eight in flight per thread,
+ * enqueued on `stream`; the caller times it with events.  The ruler walks are
+ * chains of random accesses, and this is the rate they are compared with.
+ * `sink` is one device word; it is written only if the words a thread read
+ * xor to one particular value (so that the reads cannot be dropped).
+ */
+int benes_probe_gather(const uint32_t *table, int log2_words, size_t gathers, uint32_t *sink,
+                       benes_stream_t stream);
 
 /* Largest block size (log2) finished inside one CTA by the fused kernel. */
 int benes_fused_log2m(void);

@@ -52,6 +52,8 @@ SYMBOLS = {
     "benes_profile_span": (_i, [_i, ctypes.POINTER(_i), ctypes.POINTER(ctypes.c_ulonglong),
                                 ctypes.POINTER(ctypes.c_double)]),
     "benes_profile_kind_name": (ctypes.c_char_p, [_i]),
+    "benes_shard_batch": (_i, [_i, _i, _i, ctypes.POINTER(_i), ctypes.POINTER(_i)]),
+    "benes_probe_gather": (_i, [_vp, _i, _sz, _vp, _vp]),
     "benes_fused_log2m": (_i, []),
     "benes_status_string": (ctypes.c_char_p, [_i]),
 }
@@ -258,6 +260,19 @@ def benes_profile_spans():
 
 def benes_profile_kind_name(kind: int) -> str:
     return load().benes_profile_kind_name(kind).decode()
+
+
+def benes_shard_batch(batch: int, world: int, rank: int):
+    """(first, count): the contiguous slice of a batch that rank `rank` of `world` routes."""
+    first, count = _i(0), _i(0)
+    _check(load().benes_shard_batch(batch, world, rank, ctypes.byref(first), ctypes.byref(count)),
+           "benes_shard_batch")
+    return first.value, count.value
+
+
+def benes_probe_gather(table: torch.Tensor, log2_words: int, gathers: int, sink: torch.Tensor, stream=None) -> None:
+    _check(load().benes_probe_gather(_dev_ptr(table, "table"), log2_words, gathers, _dev_ptr(sink, "sink"),
+                                     _stream(stream)), "benes_probe_gather")
 
 
 def benes_fused_log2m() -> int:

@@ -12,7 +12,6 @@ namespace benes {
 namespace {
 
 constexpr int kThreads = 256;
-constexpr int kSMs = 148;
 
 template <typename E> struct Pair;
 template <> struct Pair<uint32_t> { using type = uint2; };
@@ -62,7 +61,7 @@ int launch_typed(const uint32_t *bits, const void *x, void *y, int stage, int lo
     int level = stage <= log2n - 1 ? stage : 2 * log2n - 2 - stage;
     int log2m = log2n - level;
     size_t blocks = (switches + kThreads - 1) / kThreads;
-    size_t cap = size_t(kSMs) * 16;
+    size_t cap = size_t(sm_count()) * 16;
     int grid = int(blocks < cap ? blocks : cap);
     if (stage <= log2n - 1)
         k_apply_stage<E, 0><<<grid, kThreads, 0, s>>>(bits, static_cast<const E *>(x),

@@ -255,11 +255,14 @@ int apply_fused_typed(const uint32_t *bits, const E *in, E *out, E *scratch, int
     // elements fit one SM, so that one CTA's copies overlap the others' stages
     const size_t smem_outer = size_t(kSmemElems) * sizeof(E) + size_t(7) * kBitWords * 4;
     static OncePerDevice configured;
-    if (configured.first_use()) {
-        int rc;
-        if ((rc = opt_in_smem(k_apply_inner<E>, smem))) return rc;
-        if ((rc = opt_in_smem(k_apply_outer<E, false>, smem))) return rc;
-        if ((rc = opt_in_smem(k_apply_outer<E, true>, smem))) return rc;
+    {
+        const int rc0 = configured.run([&]() -> int {
+            int rc;
+            if ((rc = opt_in_smem(k_apply_inner<E>, smem))) return rc;
+            if ((rc = opt_in_smem(k_apply_outer<E, false>, smem))) return rc;
+            return opt_in_smem(k_apply_outer<E, true>, smem);
+        });
+        if (rc0) return rc0;
     }
     const int b = n < kChunkLog2 ? n : kChunkLog2;
     const int outer = n - b;                       // levels handled by the outer kernels, per side

@@ -8,8 +8,6 @@ namespace benes {
 namespace {
 
 constexpr size_t kAlign = 256;
-// Flat elements processed together by the per-level path (indices are 32 bit).
-int g_chunk_log2 = 30;
 
 struct Workspace {
     void *own = nullptr;       // library-owned buffer
@@ -21,13 +19,22 @@ struct Workspace {
 Workspace g_ws[kMaxDevices];
 std::mutex g_mu;
 
-// Tuning (benes_set_option).  kappa = 0: every loop is labelled by pointer
-// jumping over all outputs; 2..8: one ruler switch per 2^kappa switches.
-int g_kappa = 4;
-int g_walk_cap = 1 << 14;
-int g_apply_fused = 1;
-int g_inverse_partitioned = 1;
+// Tuning (benes_set_option), written and read under g_mu; an entry point works
+// on the copy it took when it was called.
+struct Options {
+    int kappa = 4;                  // 0: pointer jumping over all outputs; 2..8: one ruler switch per 2^kappa
+    int walk_cap = 1 << 14;
+    int apply_fused = 1;
+    int inverse_partitioned = 1;
+    int chunk_log2 = 30;            // flat elements processed together by the per-level path (indices are 32 bit)
+};
+Options g_opt;
 constexpr int kMaxLevels = 32;
+
+Options options() {
+    std::lock_guard<std::mutex> lk(g_mu);
+    return g_opt;
+}
 
 inline size_t align_up(size_t v) { return (v + kAlign - 1) & ~(kAlign - 1); }
 
@@ -68,8 +75,8 @@ inline bool bad_shape(int log2n, int batch) {
 inline size_t stage_words(int log2n) { return log2n >= 6 ? (size_t(1) << (log2n - 6)) : 1; }
 
 // permutations per chunk of the per-level path
-inline size_t level_chunk(int log2n, size_t batch) {
-    size_t per = (size_t(1) << g_chunk_log2) >> log2n;
+inline size_t level_chunk(int log2n, size_t batch, int chunk_log2) {
+    size_t per = (size_t(1) << chunk_log2) >> log2n;
     if (per < 1) per = 1;
     return batch < per ? batch : per;
 }
@@ -80,7 +87,7 @@ inline size_t level_chunk(int log2n, size_t batch) {
 constexpr int kMaxKappa = 8, kMinKappa = 2;
 size_t route_ws_bytes(int log2n, size_t batch) {
     if (log2n <= kFusedLog2M) return 0;
-    size_t T = level_chunk(log2n, batch) << log2n;
+    size_t T = level_chunk(log2n, batch, options().chunk_log2) << log2n;
     return 2 * align_up(T * 8) + 2 * align_up(T * 4) + align_up(T * 8) +
            align_up(sampled_scratch_bytes(T, kMinKappa)) + align_up(kMaxLevels * 4) +
            align_up(kInverseMaxBuckets * 4);
@@ -97,7 +104,6 @@ size_t apply_ws_bytes(int elem_bytes, int log2n, size_t batch) {
 // copied to the host on the side stream while the next levels run.
 constexpr int kMaxPieces = 8;
 static_assert(kMaxPieces >= kApplyMaxParts, "the host pipe's events serve the apply parts too");
-constexpr int kFusedSplitWave = 148;   // CTAs of the fused kernel that run together (one per SM)
 struct HostPipe {
     uint32_t *bits_host = nullptr;     // finished stages go here (same layout as `bits`)
     cudaStream_t side = nullptr;
@@ -118,8 +124,9 @@ int copy_stage_rows(const HostPipe &hp, const uint32_t *bits, int n, size_t batc
 
 // The levels whose blocks exceed the in-CTA size in HBM, then the fused tail.
 int route_levels(const uint32_t *perm, int n, size_t batch, uint32_t *bits, char *ws, cudaStream_t s,
-                 const HostPipe *hp = nullptr) {
+                 const Options &opt, const HostPipe *hp = nullptr) {
     const size_t T = batch << n;
+    const size_t kFusedSplitWave = size_t(sm_count());   // CTAs of the fused kernel that run together (one per SM)
     void *Sbuf[2];                     // two generations of switch records (wide: 16 B per switch)
     uint32_t *Qbuf[2];
     size_t off = 0;
@@ -129,12 +136,13 @@ int route_levels(const uint32_t *perm, int n, size_t batch, uint32_t *bits, char
     Qbuf[1] = reinterpret_cast<uint32_t *>(ws + off); off += align_up(T * 4);
     unsigned long long *Wd = reinterpret_cast<unsigned long long *>(ws + off); off += align_up(T * 8);
     char *sampled = ws + off; off += align_up(sampled_scratch_bytes(T, kMinKappa));
+    // per level: a gate, raised by a walk that gave up
     uint32_t *gates = reinterpret_cast<uint32_t *>(ws + off); off += align_up(kMaxLevels * 4);
     uint32_t *fill = reinterpret_cast<uint32_t *>(ws + off);
     // Small inputs are bound by the longest walk of a level, not by throughput:
     // closer rulers (shorter walks) pay there although the lists get longer.
-    const int kappa = (g_kappa > 3 && T <= (size_t(1) << 22)) ? 3 : g_kappa;
-    const uint32_t cap = uint32_t(g_walk_cap);
+    const int kappa = (opt.kappa > 3 && T <= (size_t(1) << 22)) ? 3 : opt.kappa;
+    const uint32_t cap = uint32_t(opt.walk_cap);
     SampledScratch sc;
     int rc;
     if (kappa) {
@@ -148,7 +156,7 @@ int route_levels(const uint32_t *perm, int n, size_t batch, uint32_t *bits, char
         ProfileScope ps(kInverse, s);
         // the 64-bit word array is free until the first level is labelled
         // (the bucketed form needs whole buckets, of 2^18 entries at most)
-        const bool bucketed = g_inverse_partitioned && T >= (size_t(1) << kInversePartitionMinLog2) &&
+        const bool bucketed = opt.inverse_partitioned && T >= (size_t(1) << kInversePartitionMinLog2) &&
                               (T & ((size_t(1) << 18) - 1)) == 0;
         const int pieces = hp ? hp->pieces : 0;
         const bool pk = rec_is_packed(n, kappa);
@@ -212,7 +220,7 @@ int route_levels(const uint32_t *perm, int n, size_t batch, uint32_t *bits, char
     const size_t blocks = T >> fused_m;
     // the stages of the in-CTA levels are one run of rows in the middle
     const int first = n - fused_m, rows = 2 * fused_m - 1;
-    if (hp && hp->bits_host && batch == 1 && blocks >= 4 * size_t(kFusedSplitWave)) {
+    if (hp && hp->bits_host && batch == 1 && blocks >= 4 * kFusedSplitWave) {
         // Two launches of whole waves of CTAs (one CTA per SM): the columns the
         // first one has finished go to the host while the second one runs.
         const size_t waves = (blocks + kFusedSplitWave - 1) / kFusedSplitWave;
@@ -334,12 +342,13 @@ int benes_route(const uint32_t *perm, int log2n, int batch, uint32_t *switch_bit
     void *ws = nullptr;
     int rc = get_workspace(route_ws_bytes(n, size_t(batch)), &ws);
     if (rc) return rc;
-    const size_t chunk = level_chunk(n, size_t(batch));
+    const Options opt = options();
+    const size_t chunk = level_chunk(n, size_t(batch), opt.chunk_log2);
     for (size_t b0 = 0; b0 < size_t(batch); b0 += chunk) {
         size_t nb = size_t(batch) - b0 < chunk ? size_t(batch) - b0 : chunk;
         rc = route_levels(perm + (b0 << n), n, nb,
                           switch_bits + b0 * size_t(2 * n - 1) * stage_words(n),
-                          static_cast<char *>(ws), s);
+                          static_cast<char *>(ws), s, opt);
         if (rc) return rc;
     }
     return BENES_OK;
@@ -357,7 +366,7 @@ int benes_apply_ex(const uint32_t *switch_bits, const void *in, void *out, int e
         int rc = get_workspace(apply_ws_bytes(elem_bytes, n, size_t(batch)), &ws);
         if (rc) return rc;
     }
-    if (g_apply_fused) {
+    if (options().apply_fused) {
         ProfileScope ps(kApplyFused, s);
         return launch_apply_fused(switch_bits, in, out, ws, elem_bytes, n, size_t(batch), s);
     }
@@ -441,7 +450,8 @@ int benes_route_host(const uint32_t *perm_host, int log2n, int batch, uint32_t *
     uint32_t *d_perm = reinterpret_cast<uint32_t *>(base + align_up(inner));
     uint32_t *d_bits = reinterpret_cast<uint32_t *>(base + align_up(inner) + align_up(perm_bytes));
     const int n = log2n;
-    if (n > kFusedLog2M && level_chunk(n, size_t(batch)) == size_t(batch)) {
+    const Options opt = options();
+    if (n > kFusedLog2M && level_chunk(n, size_t(batch), opt.chunk_log2) == size_t(batch)) {
         // one chunk: copies overlapped with the levels (see HostPipe)
         HostPipe *hp = nullptr;
         if ((rc = host_pipe_for_current_device(&hp))) return rc;
@@ -458,7 +468,7 @@ int benes_route_host(const uint32_t *perm_host, int log2n, int batch, uint32_t *
                                            cudaMemcpyHostToDevice, hp->side));
             BENES_CUDA_TRY(cudaEventRecord(hp->piece_ready[i], hp->side));
         }
-        rc = route_levels(d_perm, n, size_t(batch), d_bits, base, s, hp);
+        rc = route_levels(d_perm, n, size_t(batch), d_bits, base, s, opt, hp);
         cudaError_t e1 = cudaStreamSynchronize(hp->side), e2 = cudaStreamSynchronize(s);
         if (rc) return rc;
         return (e1 == cudaSuccess && e2 == cudaSuccess) ? BENES_OK : BENES_ERR_CUDA;
@@ -488,7 +498,7 @@ int benes_apply_host(const uint32_t *switch_bits_host, const void *in_host, void
     uint32_t *d_bits = reinterpret_cast<uint32_t *>(d_out + align_up(data_bytes));
     BENES_CUDA_TRY(cudaMemcpyAsync(d_bits, switch_bits_host, bits_bytes, cudaMemcpyHostToDevice, s));
     const size_t chunks = apply_fused_chunks(log2n, size_t(batch));
-    if (g_apply_fused && data_bytes >= (size_t(1) << 26) && chunks % kApplyMaxParts == 0 && chunks > 0) {
+    if (options().apply_fused && data_bytes >= (size_t(1) << 26) && chunks % kApplyMaxParts == 0 && chunks > 0) {
         // The payload arrives in parts on the side stream, behind the switch words:
         // the first pass starts on a part as soon as it is there, and the parts the
         // last pass has finished leave on the side stream while it still runs.
@@ -550,23 +560,23 @@ int benes_set_option(int key, int value) {
     switch (key) {
         case BENES_OPT_SAMPLE_LOG2K:
             if (value != 0 && (value < kMinKappa || value > kMaxKappa)) return BENES_ERR_BADARG;
-            g_kappa = value;
+            g_opt.kappa = value;
             return BENES_OK;
         case BENES_OPT_WALK_CAP:
             if (value < 1 || value > (1 << 24)) return BENES_ERR_BADARG;
-            g_walk_cap = value;
+            g_opt.walk_cap = value;
             return BENES_OK;
         case BENES_OPT_APPLY_FUSED:
             if (value != 0 && value != 1) return BENES_ERR_BADARG;
-            g_apply_fused = value;
+            g_opt.apply_fused = value;
             return BENES_OK;
         case BENES_OPT_INVERSE_PARTITIONED:
             if (value != 0 && value != 1) return BENES_ERR_BADARG;
-            g_inverse_partitioned = value;
+            g_opt.inverse_partitioned = value;
             return BENES_OK;
         case BENES_OPT_CHUNK_LOG2:
             if (value < 16 || value > 30) return BENES_ERR_BADARG;
-            g_chunk_log2 = value;
+            g_opt.chunk_log2 = value;
             return BENES_OK;
         default: return BENES_ERR_BADARG;
     }
@@ -575,11 +585,11 @@ int benes_set_option(int key, int value) {
 int benes_get_option(int key) {
     std::lock_guard<std::mutex> lk(g_mu);
     switch (key) {
-        case BENES_OPT_SAMPLE_LOG2K: return g_kappa;
-        case BENES_OPT_WALK_CAP: return g_walk_cap;
-        case BENES_OPT_APPLY_FUSED: return g_apply_fused;
-        case BENES_OPT_INVERSE_PARTITIONED: return g_inverse_partitioned;
-        case BENES_OPT_CHUNK_LOG2: return g_chunk_log2;
+        case BENES_OPT_SAMPLE_LOG2K: return g_opt.kappa;
+        case BENES_OPT_WALK_CAP: return g_opt.walk_cap;
+        case BENES_OPT_APPLY_FUSED: return g_opt.apply_fused;
+        case BENES_OPT_INVERSE_PARTITIONED: return g_opt.inverse_partitioned;
+        case BENES_OPT_CHUNK_LOG2: return g_opt.chunk_log2;
         default: return BENES_ERR_BADARG;
     }
 }

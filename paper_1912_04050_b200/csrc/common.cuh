@@ -5,6 +5,9 @@
 #include <stdint.h>
 #include <stddef.h>
 
+#include <atomic>
+#include <mutex>
+
 #include "benes.h"
 
 namespace benes {
@@ -26,7 +29,10 @@ extern unsigned long long g_launches;
 #define BENES_CUDA_TRY(expr)                                   \
     do {                                                       \
         cudaError_t e_ = (expr);                               \
-        if (e_ != cudaSuccess) return BENES_ERR_CUDA;          \
+        if (e_ != cudaSuccess) {                               \
+            cudaGetLastError(); /* reported here, not by a later launch */ \
+            return BENES_ERR_CUDA;                             \
+        }                                                      \
     } while (0)
 
 // Result of the launch just issued; a launch error is taken off the runtime's
@@ -40,16 +46,24 @@ inline int launch_status() {
 // them the first time it runs on each device of the process.
 constexpr int kMaxDevices = 64;
 struct OncePerDevice {
+    std::mutex mu;
     bool done[kMaxDevices] = {};
-    // true if the caller still has to configure the current device
-    bool first_use() {
+    // Runs `configure` (returns a status) the first time on each device; a second
+    // thread that arrives meanwhile waits until the attributes are set.
+    template <class F>
+    int run(F &&configure) {
         int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return true;
-        if (done[dev]) return false;
-        done[dev] = true;
-        return true;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return BENES_ERR_CUDA; }
+        std::lock_guard<std::mutex> lk(mu);
+        if (done[dev]) return BENES_OK;
+        const int rc = configure();
+        if (rc == BENES_OK) done[dev] = true;
+        return rc;
     }
 };
+
+// Multiprocessors of the current device (read once per device).
+int sm_count();
 
 // Optional event timing of a group of launches of one kind (see benes.h).
 enum ProfileKind {
@@ -162,9 +176,9 @@ __device__ __forceinline__ unsigned long long make_word(uint32_t nxt, uint32_t m
 }
 
 // The streaming kernels of a level give every CTA `rounds` consecutive groups of
-// `threads` items: as many as keep 8 CTAs per SM of a 148-SM part busy, at most 16.
+// `threads` items: as many as keep 8 CTAs per SM busy, at most 16.
 inline uint32_t stream_rounds(size_t items, int threads) {
-    const size_t r = items / (size_t(threads) * 148 * 8);
+    const size_t r = items / (size_t(threads) * size_t(sm_count()) * 8);
     return uint32_t(r < 1 ? 1 : (r > 16 ? 16 : r));
 }
 

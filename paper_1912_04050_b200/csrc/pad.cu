@@ -8,11 +8,10 @@ namespace benes {
 namespace {
 
 constexpr int kThreads = 256;
-constexpr int kSMs = 148;
 
 inline unsigned grid_for(size_t items) {
     size_t blocks = (items + kThreads - 1) / kThreads;
-    size_t cap = size_t(kSMs) * 16;
+    size_t cap = size_t(sm_count()) * 16;
     return unsigned(blocks < cap ? (blocks ? blocks : 1) : cap);
 }
 
@@ -118,7 +117,7 @@ int launch_export_butterfly(const uint32_t *bits, uint32_t *out, int log2n, size
     const size_t rows = batch * size_t(2 * log2n - 1);
     const size_t total = rows * words * 32;
     size_t blocks = (total + 255) / 256;
-    if (blocks > size_t(kSMs) * 16) blocks = size_t(kSMs) * 16;
+    if (blocks > size_t(sm_count()) * 16) blocks = size_t(sm_count()) * 16;
     k_export_butterfly<<<unsigned(blocks), 256, 0, s>>>(bits, out, log2n, rows, words);
     return launch_status();
 }

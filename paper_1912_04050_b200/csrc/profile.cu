@@ -11,17 +11,19 @@ struct Span {
     int kind;
     cudaEvent_t start, stop;
     unsigned long long launches;
+    int dev;                        // the device the events were created on
 };
 
 bool g_enabled = false;
 std::vector<Span> g_spans;          // spans recorded since the last reset
-std::vector<cudaEvent_t> g_pool;    // events free for reuse
+std::vector<cudaEvent_t> g_pool[kMaxDevices];    // events free for reuse, per device (an event belongs to one)
 std::mutex g_pmu;
 
-cudaEvent_t take_event() {
-    if (!g_pool.empty()) {
-        cudaEvent_t e = g_pool.back();
-        g_pool.pop_back();
+cudaEvent_t take_event(int dev) {
+    std::vector<cudaEvent_t> &pool = g_pool[dev];
+    if (!pool.empty()) {
+        cudaEvent_t e = pool.back();
+        pool.pop_back();
         return e;
     }
     cudaEvent_t e = nullptr;
@@ -37,10 +39,12 @@ const char *kNames[BENES_PROFILE_KINDS] = {"inverse", "full_label", "split", "fu
 
 ProfileScope::ProfileScope(int kind, cudaStream_t s) : kind_(kind), s_(s), slot_(-1), launches0_(g_launches) {
     if (!g_enabled) return;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return; }
     std::lock_guard<std::mutex> lk(g_pmu);
-    Span sp{kind, take_event(), take_event(), 0};
+    Span sp{kind, take_event(dev), take_event(dev), 0, dev};
     if (!sp.start || !sp.stop) return;
-    cudaEventRecord(sp.start, s);
+    if (cudaEventRecord(sp.start, s) != cudaSuccess) { cudaGetLastError(); return; }
     g_spans.push_back(sp);
     slot_ = int(g_spans.size()) - 1;
 }
@@ -49,7 +53,7 @@ ProfileScope::~ProfileScope() {
     if (slot_ < 0) return;
     std::lock_guard<std::mutex> lk(g_pmu);
     if (slot_ >= int(g_spans.size())) return;
-    cudaEventRecord(g_spans[slot_].stop, s_);
+    if (cudaEventRecord(g_spans[slot_].stop, s_) != cudaSuccess) cudaGetLastError();
     g_spans[slot_].launches = g_launches - launches0_;
 }
 
@@ -69,8 +73,8 @@ int benes_profile_reset(void) {
     std::lock_guard<std::mutex> lk(g_pmu);
     for (Span &sp : g_spans) {
         cudaEventSynchronize(sp.stop);
-        g_pool.push_back(sp.start);
-        g_pool.push_back(sp.stop);
+        g_pool[sp.dev].push_back(sp.start);
+        g_pool[sp.dev].push_back(sp.stop);
     }
     g_spans.clear();
     return BENES_OK;

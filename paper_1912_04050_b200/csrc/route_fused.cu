@@ -363,13 +363,17 @@ int launch_one(const uint32_t *P, int records, size_t first_block, size_t blocks
                cudaStream_t s) {
     using C = FusedCfg<LOGM>;
     static OncePerDevice configured;
-    if (C::kSmemBytes > 48 * 1024 && configured.first_use()) {
-        BENES_CUDA_TRY(cudaFuncSetAttribute(k_route_fused<LOGM>,
-                                            cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            int(C::kSmemBytes)));
-        BENES_CUDA_TRY(cudaFuncSetAttribute(k_route_fused<LOGM>,
-                                            cudaFuncAttributePreferredSharedMemoryCarveout,
-                                            cudaSharedmemCarveoutMaxShared));
+    if (C::kSmemBytes > 48 * 1024) {
+        const int rc = configured.run([]() -> int {
+            BENES_CUDA_TRY(cudaFuncSetAttribute(k_route_fused<LOGM>,
+                                                cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                int(C::kSmemBytes)));
+            BENES_CUDA_TRY(cudaFuncSetAttribute(k_route_fused<LOGM>,
+                                                cudaFuncAttributePreferredSharedMemoryCarveout,
+                                                cudaSharedmemCarveoutMaxShared));
+            return BENES_OK;
+        });
+        if (rc) return rc;
     }
     k_route_fused<LOGM><<<unsigned(blocks), C::kThreads, C::kSmemBytes, s>>>(P, records, bits, log2n,
                                                                              uint32_t(first_block));

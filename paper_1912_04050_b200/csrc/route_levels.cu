@@ -19,20 +19,36 @@
 
 #include <cooperative_groups.h>
 
+#include <atomic>
+
 namespace cg = cooperative_groups;
 
 namespace benes {
 
 unsigned long long g_launches = 0;
 
+int sm_count() {
+    static std::atomic<int> cached[kMaxDevices] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 148;
+    int v = cached[dev].load(std::memory_order_relaxed);
+    if (v == 0) {
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v < 1) {
+            cudaGetLastError();
+            v = 148;
+        }
+        cached[dev].store(v, std::memory_order_relaxed);
+    }
+    return v;
+}
+
 namespace {
 
 constexpr int kThreads = 256;
-constexpr int kSMs = 148;
 
 inline int grid_for(size_t work_items, int per_sm = 8) {
     size_t blocks = (work_items + kThreads - 1) / kThreads;
-    size_t cap = size_t(kSMs) * per_sm;
+    size_t cap = size_t(sm_count()) * per_sm;
     return int(blocks < cap ? (blocks ? blocks : 1) : cap);
 }
 
@@ -378,12 +394,16 @@ int launch_inverse_partition_piece(const uint32_t *perm, void *S, bool packed, v
     const unsigned grid = unsigned(count / kPartChunk);
     const size_t smem = partition_smem(buckets);
     static OncePerDevice configured;
-    if (configured.first_use()) {
-        const int most = int(partition_smem(kInverseMaxBuckets));
-        BENES_CUDA_TRY(cudaFuncSetAttribute(k_inverse_partition<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most));
-        BENES_CUDA_TRY(cudaFuncSetAttribute(k_inverse_partition<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, most));
-        BENES_CUDA_TRY(cudaFuncSetAttribute(k_inverse_scatter_smem, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            4 << kBucketSmemLog2));
+    {
+        const int rc = configured.run([]() -> int {
+            const int most = int(partition_smem(kInverseMaxBuckets));
+            BENES_CUDA_TRY(cudaFuncSetAttribute(k_inverse_partition<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most));
+            BENES_CUDA_TRY(cudaFuncSetAttribute(k_inverse_partition<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, most));
+            BENES_CUDA_TRY(cudaFuncSetAttribute(k_inverse_scatter_smem, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                4 << kBucketSmemLog2));
+            return BENES_OK;
+        });
+        if (rc) return rc;
     }
     if (packed)
         k_inverse_partition<true><<<grid, kPartThreads, smem, s>>>(

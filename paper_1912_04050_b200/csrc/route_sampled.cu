@@ -321,9 +321,13 @@ template <int PER>
 int launch_list_label(unsigned long long *W, uint32_t count, int beta, uint32_t *cb, cudaStream_t s) {
     static OncePerDevice configured;
     const size_t smem = (size_t(1) << beta) * 8;
-    if (configured.first_use()) {
-        BENES_CUDA_TRY(cudaFuncSetAttribute(k_list_label<PER>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            (1 << kListSmemLog2) * 8));
+    {
+        const int rc = configured.run([]() -> int {
+            BENES_CUDA_TRY(cudaFuncSetAttribute(k_list_label<PER>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                (1 << kListSmemLog2) * 8));
+            return BENES_OK;
+        });
+        if (rc) return rc;
     }
     k_list_label<PER><<<count >> beta, (1u << beta) / PER, smem, s>>>(W, beta, cb);
     return launch_status();
@@ -376,9 +380,14 @@ k_list_label_rec(const uint4 *__restrict__ rec, uint32_t *__restrict__ cb, int l
 template <int PER>
 int launch_list_label_rec(const uint4 *rec, uint32_t *cb, uint32_t count, int beta, int m, cudaStream_t s) {
     static OncePerDevice configured;
-    if (configured.first_use())
-        BENES_CUDA_TRY(cudaFuncSetAttribute(k_list_label_rec<PER>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            (1 << kListSmemLog2) * 4));
+    {
+        const int rc = configured.run([]() -> int {
+            BENES_CUDA_TRY(cudaFuncSetAttribute(k_list_label_rec<PER>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                (1 << kListSmemLog2) * 4));
+            return BENES_OK;
+        });
+        if (rc) return rc;
+    }
     k_list_label_rec<PER><<<count >> beta, (1u << beta) / PER, (size_t(1) << beta) * 4, s>>>(rec, cb, beta, m);
     return launch_status();
 }

@@ -9,6 +9,7 @@ import socket
 import sys
 
 import numpy as np
+import pytest
 import torch
 import torch.distributed as dist
 import torch.multiprocessing as mp
@@ -68,3 +69,46 @@ def test_job_value_counts_every_replica():
     import bench
     assert bench.whole_job_value(1 << 20, 1, 2.0) == (1 << 20) / 2e-3
     assert bench.whole_job_value(1 << 20, 8, 2.0) == 8 * (1 << 20) / 2e-3
+
+
+def test_plain_start_with_gpus_2_spawns_two_ranks():
+    """`python bench.py --gpus 2` without torchrun's variables must start the two ranks itself;
+    driven here through the CPU rank check (gloo): one line, n_gpus = 2, the slowest rank's
+    time, every replica counted, a different permutation on each rank."""
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items()
+           if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_ADDR", "MASTER_PORT")}
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--rank-check",
+                          "--workload", "c1"], env=env, capture_output=True, text=True, timeout=300)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [ln for ln in out.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1
+    line = json.loads(lines[0])
+    assert line["n_gpus"] == 2 and line["ms_per_step"] == 2.0
+    assert line["value"] == 2 * (1 << 10) / 2e-3
+    assert len(set(line["rank_inputs"])) == 2
+
+
+def test_gpus_must_match_the_world_size():
+    import subprocess
+    env = dict(os.environ, RANK="0", LOCAL_RANK="0", WORLD_SIZE="1", MASTER_ADDR="127.0.0.1",
+               MASTER_PORT=str(_free_port()))
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--rank-check",
+                          "--workload", "c1"], env=env, capture_output=True, text=True, timeout=300)
+    assert out.returncode != 0 and "WORLD_SIZE" in out.stderr
+
+
+def test_batch_slices_cover_the_batch_once():
+    from paper_1912_04050_b200 import binding, build
+    build.build()
+    for batch, world in ((16384, 8), (5, 8), (7, 3), (1, 1), (1000, 7)):
+        slices = [binding.benes_shard_batch(batch, world, r) for r in range(world)]
+        assert slices[0][0] == 0
+        for (f0, c0), (f1, _) in zip(slices, slices[1:]):
+            assert f1 == f0 + c0
+        assert slices[-1][0] + slices[-1][1] == batch
+        counts = [c for _, c in slices]
+        assert max(counts) - min(counts) <= 1
+    with pytest.raises(binding.BenesError):
+        binding.benes_shard_batch(4, 2, 2)
