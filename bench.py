@@ -518,6 +518,9 @@ def run_gpu(args):
     if args.kappa is not None:
         binding.benes_set_option(binding.OPT_SAMPLE_LOG2K, args.kappa)
 
+    if args.cluster is not None:
+        binding.benes_set_option(binding.OPT_CLUSTER, args.cluster)
+
     name = args.workload
     stream = torch.cuda.Stream()
     case = GpuCase(name, rank, stream)
@@ -692,6 +695,8 @@ def main():
     ap.add_argument("--no-side-workloads", action="store_true")
     ap.add_argument("--kappa", type=int, default=None,
                     help="ruler spacing (log2) of the loop labelling; 0 = full pointer jumping")
+    ap.add_argument("--cluster", type=int, default=None,
+                    help="1: blocks of 2^16 finished by clusters of two CTAs; 0: blocks of 2^15 in one CTA")
     ap.add_argument("--rank-check", action="store_true",
                     help="run only the rank plumbing on the CPU (gloo); used by the tests")
     args = ap.parse_args()

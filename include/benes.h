@@ -203,6 +203,10 @@ int benes_validate_perm(const uint32_t *perm, int log2n, int batch, benes_stream
  *   BENES_OPT_CHUNK_LOG2 : 16..30 (default 30): a batch whose levels do not fit one
  *       CTA is processed in chunks of at most 2^value elements (whole
  *       permutations, at least one); bounds the workspace of a large batch.
+ *   BENES_OPT_CLUSTER : 1 = blocks of 2^16 outputs (whole permutations of N = 2^16,
+ *       and the tail of larger ones) are finished by a thread-block cluster of two
+ *       CTAs over distributed shared memory instead of one more level in global
+ *       memory; 0 = blocks of 2^15 in one CTA.  Same result.
  * benes_set_option returns BENES_OK or BENES_ERR_BADARG; benes_get_option
  * returns the value, or BENES_ERR_BADARG for an unknown key.
  */
@@ -211,6 +215,7 @@ int benes_validate_perm(const uint32_t *perm, int log2n, int batch, benes_stream
 #define BENES_OPT_APPLY_FUSED 2
 #define BENES_OPT_INVERSE_PARTITIONED 3
 #define BENES_OPT_CHUNK_LOG2 4
+#define BENES_OPT_CLUSTER 5
 int benes_set_option(int key, int value);
 int benes_get_option(int key);
 
@@ -261,6 +266,21 @@ int benes_shard_batch(int batch, int world, int rank, int *first, int *count);
  */
 int benes_probe_gather(const uint32_t *table, int log2_words, size_t gathers, uint32_t *sink,
                        benes_stream_t stream);
+
+/*
+ * Checked build.  Every index a kernel forms from data is forced into range (a
+ * mask or a clamp), which is what keeps a non-permutation input memory-safe; on a
+ * permutation no such guard ever changes its value.  The library built with
+ * -DBENES_DEBUG (libbenes_debug.so, same ABI) counts, in device words, every guard
+ * that did change a value, and remembers the source line of one of them.  Nothing
+ * traps and nothing is printed.  benes_debug_build returns 1 for that build, 0
+ * otherwise.  benes_debug_guard_hits synchronises the current device, stores the
+ * number of such events since the last clearing in *hits (always 0 in the normal
+ * build), writes "file:line" of one of them to `where` (may be NULL) and clears
+ * the counters if `clear` is non-zero.
+ */
+int benes_debug_build(void);
+int benes_debug_guard_hits(unsigned long long *hits, char *where, size_t where_bytes, int clear);
 
 /* Largest block size (log2) finished inside one CTA by the fused kernel. */
 int benes_fused_log2m(void);

@@ -54,6 +54,8 @@ SYMBOLS = {
     "benes_profile_kind_name": (ctypes.c_char_p, [_i]),
     "benes_shard_batch": (_i, [_i, _i, _i, ctypes.POINTER(_i), ctypes.POINTER(_i)]),
     "benes_probe_gather": (_i, [_vp, _i, _sz, _vp, _vp]),
+    "benes_debug_build": (_i, []),
+    "benes_debug_guard_hits": (_i, [ctypes.POINTER(ctypes.c_ulonglong), ctypes.c_char_p, _sz, _i]),
     "benes_fused_log2m": (_i, []),
     "benes_status_string": (ctypes.c_char_p, [_i]),
 }
@@ -67,20 +69,31 @@ class BenesError(RuntimeError):
         super().__init__("%s failed: %s (%d)" % (what, status_string(status), status))
 
 
+def _open(path: str) -> ctypes.CDLL:
+    if not os.path.exists(path):
+        raise RuntimeError(
+            "%s is not built (%s); run `python -m paper_1912_04050_b200.build`. "
+            "There is no CPU fallback." % (os.path.basename(path), path))
+    lib = ctypes.CDLL(path)
+    for name, (res, args) in SYMBOLS.items():
+        fn = getattr(lib, name)
+        fn.restype, fn.argtypes = res, args
+    return lib
+
+
 def load() -> ctypes.CDLL:
     """Load the CUDA library; fails loudly if it is not built."""
     global _lib
     if _lib is None:
-        if not os.path.exists(LIB_PATH):
-            raise RuntimeError(
-                "libbenes.so is not built (%s); run `python -m paper_1912_04050_b200.build`. "
-                "There is no CPU fallback." % LIB_PATH)
-        lib = ctypes.CDLL(LIB_PATH)
-        for name, (res, args) in SYMBOLS.items():
-            fn = getattr(lib, name)
-            fn.restype, fn.argtypes = res, args
-        _lib = lib
+        _lib = _open(LIB_PATH)
     return _lib
+
+
+def use_library(path: str = None) -> None:
+    """Route every call of this module through another build of the library with the same
+    ABI (the checked build, libbenes_debug.so); None switches back to libbenes.so."""
+    global _lib
+    _lib = _open(path or LIB_PATH)
 
 
 def status_string(status: int) -> str:
@@ -220,6 +233,7 @@ OPT_WALK_CAP = 1
 OPT_APPLY_FUSED = 2
 OPT_INVERSE_PARTITIONED = 3
 OPT_CHUNK_LOG2 = 4
+OPT_CLUSTER = 5
 
 
 def benes_set_option(key: int, value: int) -> None:
@@ -273,6 +287,19 @@ def benes_shard_batch(batch: int, world: int, rank: int):
 def benes_probe_gather(table: torch.Tensor, log2_words: int, gathers: int, sink: torch.Tensor, stream=None) -> None:
     _check(load().benes_probe_gather(_dev_ptr(table, "table"), log2_words, gathers, _dev_ptr(sink, "sink"),
                                      _stream(stream)), "benes_probe_gather")
+
+
+def benes_debug_build() -> bool:
+    return bool(load().benes_debug_build())
+
+
+def benes_debug_guard_hits(clear: bool = True):
+    """(events, "file:line" of one of them): index guards that had to change a value."""
+    hits = ctypes.c_ulonglong(0)
+    where = ctypes.create_string_buffer(128)
+    _check(load().benes_debug_guard_hits(ctypes.byref(hits), where, 128, 1 if clear else 0),
+           "benes_debug_guard_hits")
+    return hits.value, where.value.decode()
 
 
 def benes_fused_log2m() -> int:

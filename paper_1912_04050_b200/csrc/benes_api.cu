@@ -2,9 +2,26 @@
 // workspace management and the host-side level loop.
 #include "common.cuh"
 
+#include <cstdio>
 #include <mutex>
+#include <vector>
 
 namespace benes {
+
+#ifdef BENES_DEBUG
+namespace {
+struct GuardEntry {
+    GuardReader read;
+    const char *file;
+};
+std::vector<GuardEntry> &guard_registry() {
+    static std::vector<GuardEntry> entries;       // filled by static constructors of the kernel files
+    return entries;
+}
+}  // namespace
+void guard_register(GuardReader reader, const char *file) { guard_registry().push_back({reader, file}); }
+#endif
+
 namespace {
 
 constexpr size_t kAlign = 256;
@@ -27,6 +44,7 @@ struct Options {
     int apply_fused = 1;
     int inverse_partitioned = 1;
     int chunk_log2 = 30;            // flat elements processed together by the per-level path (indices are 32 bit)
+    int cluster = 0;                // 1: blocks of 2^16 are finished by clusters of two CTAs
 };
 Options g_opt;
 constexpr int kMaxLevels = 32;
@@ -180,7 +198,7 @@ int route_levels(const uint32_t *perm, int n, size_t batch, uint32_t *bits, char
     // Blocks of 2^15 are finished by one CTA each.  Up to 64 of them would leave
     // more than half of the SMs idle during the longest kernel of the route: then
     // one more level runs in HBM and twice as many CTAs finish blocks of 2^14.
-    const int fused_m = (T >> kFusedLog2M) <= 64 ? kFusedLog2M - 1 : kFusedLog2M;
+    const int fused_m = opt.cluster ? kFusedLog2M + 1 : (T >> kFusedLog2M) <= 64 ? kFusedLog2M - 1 : kFusedLog2M;
     int cur = 0;
     for (int level = 0; n - level > fused_m; ++level) {
         const int m = n - level;
@@ -339,10 +357,15 @@ int benes_route(const uint32_t *perm, int log2n, int batch, uint32_t *switch_bit
         }
         return BENES_OK;
     }
+    const Options opt = options();
+    if (n == kFusedLog2M + 1 && opt.cluster) {
+        // whole permutations of 2^16, one cluster of two CTAs each
+        ProfileScope ps(kFused, s);
+        return launch_fused(perm, 0, size_t(batch) << n, n, switch_bits, n, s);
+    }
     void *ws = nullptr;
     int rc = get_workspace(route_ws_bytes(n, size_t(batch)), &ws);
     if (rc) return rc;
-    const Options opt = options();
     const size_t chunk = level_chunk(n, size_t(batch), opt.chunk_log2);
     for (size_t b0 = 0; b0 < size_t(batch); b0 += chunk) {
         size_t nb = size_t(batch) - b0 < chunk ? size_t(batch) - b0 : chunk;
@@ -555,6 +578,33 @@ int benes_validate_perm(const uint32_t *perm, int log2n, int batch, benes_stream
 
 unsigned long long benes_launch_count(void) { return g_launches; }
 
+int benes_debug_build(void) {
+#ifdef BENES_DEBUG
+    return 1;
+#else
+    return 0;
+#endif
+}
+
+int benes_debug_guard_hits(unsigned long long *hits, char *where, size_t where_bytes, int clear) {
+    if (!hits) return BENES_ERR_BADARG;
+    *hits = 0;
+    if (where && where_bytes) where[0] = 0;
+#ifdef BENES_DEBUG
+    BENES_CUDA_TRY(cudaDeviceSynchronize());
+    for (const GuardEntry &e : guard_registry()) {
+        unsigned int w[2] = {0u, 0u};
+        const int rc = e.read(w, clear);
+        if (rc) return rc;
+        if (w[0] && where && where_bytes) std::snprintf(where, where_bytes, "%s:%u", e.file, w[1]);
+        *hits += w[0];
+    }
+#else
+    (void)clear;
+#endif
+    return BENES_OK;
+}
+
 int benes_set_option(int key, int value) {
     std::lock_guard<std::mutex> lk(g_mu);
     switch (key) {
@@ -578,6 +628,10 @@ int benes_set_option(int key, int value) {
             if (value < 16 || value > 30) return BENES_ERR_BADARG;
             g_opt.chunk_log2 = value;
             return BENES_OK;
+        case BENES_OPT_CLUSTER:
+            if (value != 0 && value != 1) return BENES_ERR_BADARG;
+            g_opt.cluster = value;
+            return BENES_OK;
         default: return BENES_ERR_BADARG;
     }
 }
@@ -590,6 +644,7 @@ int benes_get_option(int key) {
         case BENES_OPT_APPLY_FUSED: return g_opt.apply_fused;
         case BENES_OPT_INVERSE_PARTITIONED: return g_opt.inverse_partitioned;
         case BENES_OPT_CHUNK_LOG2: return g_opt.chunk_log2;
+        case BENES_OPT_CLUSTER: return g_opt.cluster;
         default: return BENES_ERR_BADARG;
     }
 }

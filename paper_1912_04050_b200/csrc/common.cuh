@@ -62,6 +62,60 @@ struct OncePerDevice {
     }
 };
 
+// ---- index guards ---------------------------------------------------------------
+// Every index a kernel forms from data is forced into range with a mask or a
+// clamp, so that an input that is not a permutation cannot cause an access out
+// of bounds.  On a permutation no guard ever changes the value it is given.  A
+// build with -DBENES_DEBUG checks exactly that: a guard that has to change its
+// value counts the event in a device word of its translation unit and keeps the
+// source line (no trap, no printf; the access itself is still the guarded one).
+// benes_debug_guard_hits adds the words up.  It stands in for a memory checker
+// where none can be run.
+//   BENES_GUARD(v, mask)          v & mask, v expected to be <= mask already
+//   BENES_GUARD16(v, mask)        the same for the low 16 bits of v (the rest is other data)
+//   BENES_GUARD_BELOW(v, n, alt)  v < n ? v : alt, v expected to be < n
+#ifdef BENES_DEBUG
+static __device__ unsigned int t_guard_words[2];         // hits, line of the last one
+__device__ __forceinline__ uint32_t guard_mask(uint32_t v, uint32_t mask, unsigned line) {
+    if (v & ~mask) {
+        atomicAdd(&t_guard_words[0], 1u);
+        t_guard_words[1] = line;
+    }
+    return v & mask;
+}
+__device__ __forceinline__ uint32_t guard_below(uint32_t v, uint32_t n, uint32_t alt, unsigned line) {
+    if (v >= n) {
+        atomicAdd(&t_guard_words[0], 1u);
+        t_guard_words[1] = line;
+        return alt;
+    }
+    return v;
+}
+#define BENES_GUARD(v, mask) ::benes::guard_mask((v), (mask), __LINE__)
+#define BENES_GUARD16(v, mask) ::benes::guard_mask((v) & 0xFFFFu, (mask), __LINE__)
+#define BENES_GUARD_BELOW(v, n, alt) ::benes::guard_below((v), (n), (alt), __LINE__)
+// Every translation unit with kernels registers a reader of its own words.
+using GuardReader = int (*)(unsigned int out[2], int clear);
+void guard_register(GuardReader reader, const char *file);
+#define BENES_GUARD_TU(name)                                                                     \
+    namespace {                                                                                  \
+    int guard_read_tu(unsigned int out[2], int clear) {                                          \
+        if (cudaMemcpyFromSymbol(out, ::benes::t_guard_words, 8) != cudaSuccess) { cudaGetLastError(); return BENES_ERR_CUDA; } \
+        if (clear) {                                                                             \
+            const unsigned int zero[2] = {0u, 0u};                                               \
+            if (cudaMemcpyToSymbol(::benes::t_guard_words, zero, 8) != cudaSuccess) { cudaGetLastError(); return BENES_ERR_CUDA; } \
+        }                                                                                        \
+        return BENES_OK;                                                                         \
+    }                                                                                            \
+    struct GuardRegistrar { GuardRegistrar() { ::benes::guard_register(&guard_read_tu, name); } } t_guard_registrar; \
+    }
+#else
+#define BENES_GUARD(v, mask) ((v) & (mask))
+#define BENES_GUARD16(v, mask) ((v) & (mask))
+#define BENES_GUARD_BELOW(v, n, alt) ((v) < (n) ? (v) : (alt))
+#define BENES_GUARD_TU(name)
+#endif
+
 // Multiprocessors of the current device (read once per device).
 int sm_count();
 
@@ -131,8 +185,8 @@ __device__ __forceinline__ void rec_read(const void *S, size_t t, int m, uint32_
     } else {
         const uint4 r = __ldcs(static_cast<const uint4 *>(S) + t);
         const uint32_t mask = (1u << m) - 1u;
-        p0 = r.x & mask;
-        p1 = r.y & mask;
+        p0 = BENES_GUARD(r.x, mask);
+        p1 = BENES_GUARD(r.y, mask);
     }
 }
 
@@ -143,7 +197,7 @@ __device__ __forceinline__ uint32_t rec_p(const void *S, uint32_t j, int m) {
         const unsigned long long w = __ldg(static_cast<const unsigned long long *>(S) + (j >> 1));
         return uint32_t(w >> ((j & 1u) ? m : 0)) & ((1u << m) - 1u);
     }
-    return static_cast<const uint32_t *>(S)[(size_t(j >> 1) << 2) | (j & 1u)] & ((1u << m) - 1u);
+    return BENES_GUARD(static_cast<const uint32_t *>(S)[(size_t(j >> 1) << 2) | (j & 1u)], (1u << m) - 1u);
 }
 
 // A thread of the streaming kernels owns the two neighbouring switches 2i and
@@ -231,7 +285,8 @@ int sampled_scratch_reset(const SampledScratch &sc, size_t total, int kappa, cud
 
 // ---- fused path (route_fused.cu) -------------------------------------------
 // Finishes levels (n - log2m) .. n-1 of every block of size 2^log2m of the flat
-// level array (total elements), one CTA per block.  log2m <= kFusedLog2M.
+// level array (total elements), one CTA per block for log2m <= kFusedLog2M, one
+// cluster of two CTAs per block for log2m = kFusedLog2M + 1.
 // P is a plain uint32 array if records == 0, wide records if 1, packed records if 2.
 // `blocks` blocks from `first_block` on (blocks = 0: all from first_block).
 int launch_fused(const void *P, int records, size_t total, int log2m, uint32_t *bits, int log2n,

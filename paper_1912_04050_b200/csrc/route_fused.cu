@@ -20,6 +20,10 @@
 // next level's P' is written afterwards.
 #include "common.cuh"
 
+#include <cooperative_groups.h>
+
+BENES_GUARD_TU("route_fused.cu")
+
 namespace benes {
 namespace {
 
@@ -48,56 +52,23 @@ __device__ __forceinline__ uint32_t fused_slot(uint32_t group, uint32_t salt) {
     return ((group + salt * 0x632BE5ABu) * 0x9E3779B1u) >> (32 - kFKappa);
 }
 
+// Levels level0 .. level0 + LOGM - 1 of the block of M = 2^LOGM outputs whose
+// sub-permutation (16-bit, local) is in Pcur.  Pnext is the other buffer of M
+// entries; `tail` = the extra scratch bytes (FusedCfg::kExtra); my_bits = where the
+// block's words of a stage start (stage_w words per stage).
 template <int LOGM>
-__global__ void __launch_bounds__(FusedCfg<LOGM>::kThreads)
-k_route_fused(const uint32_t *__restrict__ P, int records, uint32_t *__restrict__ bits, int log2n,
-              uint32_t block0) {
+__device__ __forceinline__ void fused_levels(uint16_t *Pcur, uint16_t *Pnext, uint16_t *Q, uint32_t *cw,
+                                             unsigned char *tail, uint32_t *my_bits, int n, int level0,
+                                             size_t stage_w) {
     using C = FusedCfg<LOGM>;
     constexpr int M = C::M;
     constexpr int T = C::kThreads;
     constexpr int R = C::kRulers;
     // pair loops run over a multiple of 32 so that every lane reaches the ballots
     constexpr int kPairsPadded = C::kPairs >= 32 ? C::kPairs : 32;
-
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    uint16_t *Pa = reinterpret_cast<uint16_t *>(smem_raw);
-    uint16_t *Q = Pa + M;
-    uint32_t *cw = reinterpret_cast<uint32_t *>(Q + M);
-    uint16_t *Pb = reinterpret_cast<uint16_t *>(cw + C::kColourWords);   // + scratch tail
-    // Pa and Pb swap roles every level, the labelling scratch always overlays
-    // the buffer P' is written to next; it starts at that buffer's first byte.
-    // Since only Pb is followed by the extra bytes, the scratch that does not
-    // fit into 2M bytes is taken from the tail behind Pb in both cases.
-    unsigned char *tail = reinterpret_cast<unsigned char *>(Pb + M);
-
     const int tid = threadIdx.x;
     const int lane = tid & 31;
-    const int n = log2n;
-    const int level0 = n - LOGM;               // recursion level of this CTA's block
-    const size_t flat0 = size_t(blockIdx.x + block0) << LOGM;    // a launch may cover a range of the blocks
-    // where this CTA's words of a stage start
-    const size_t N = size_t(1) << n;
-    const size_t stage_w = N >= 64 ? N / 64 : 1;
-    const size_t perm = flat0 >> n;
-    const size_t local_first_switch = (flat0 & (N - 1)) >> 1;
-    uint32_t *my_bits = bits + perm * size_t(2 * n - 1) * stage_w + (local_first_switch >> 5);
 
-    // plain array (0), wide switch records {P[2t], P[2t+1], -, -} (1), or packed
-    // records P[2t] | P[2t+1] << LOGM | ... (2)
-    for (int j = tid; j < M; j += T) {
-        size_t f = flat0 + j;
-        uint32_t v;
-        if (records == 2) {
-            const unsigned long long w = reinterpret_cast<const unsigned long long *>(P)[f >> 1];
-            v = uint32_t(w >> ((f & 1) ? LOGM : 0));
-        } else {
-            v = records ? P[((f >> 1) << 2) | (f & 1)] : P[f];
-        }
-        Pa[j] = uint16_t(v & uint32_t(M - 1));
-    }
-    __syncthreads();
-
-    uint16_t *Pcur = Pa, *Pnext = Pb;
 #pragma unroll 1
     for (int k = 0; k < LOGM; ++k) {
         const int logS = LOGM - k;
@@ -114,7 +85,7 @@ k_route_fused(const uint32_t *__restrict__ P, int records, uint32_t *__restrict_
             const size_t half_stride = stage_w * 2;
             for (int grp = tid >> 5; grp < M / 32; grp += T / 32) {
                 const int g0 = grp * 32;
-                uint32_t p = Pcur[g0 + lane] & 31u;                      // local to the 32-sub-block
+                uint32_t p = BENES_GUARD(uint32_t(Pcur[g0 + lane]), 31u);                      // local to the 32-sub-block
 #pragma unroll
                 for (int ls = 5; ls >= 2; --ls) {
                     const uint32_t sm_ = (1u << ls) - 1u, sbl = uint32_t(lane) & ~sm_;
@@ -195,7 +166,7 @@ k_route_fused(const uint32_t *__restrict__ P, int records, uint32_t *__restrict_
         // a1: block-local inverse; owners reset
         for (int j = tid; j < M; j += T) {
             uint32_t sb = uint32_t(j) & ~smask;
-            Q[sb + (Pcur[j] & smask)] = uint16_t(uint32_t(j) & smask);
+            Q[sb + BENES_GUARD(uint32_t(Pcur[j]), smask)] = uint16_t(uint32_t(j) & smask);
         }
         if (sampled)
             for (int t = tid; t < C::kPairs; t += T) own[t] = uint16_t(kNone16);
@@ -211,8 +182,8 @@ k_route_fused(const uint32_t *__restrict__ P, int records, uint32_t *__restrict_
                 uint32_t fwd = j, part = kNone16, pr = uint32_t(rho) ^ 1u;
                 if (!side0) own[t0] = uint16_t(rho << 1);
                 uint32_t pp = *reinterpret_cast<const uint32_t *>(Pcur + 2u * t0);
-                uint32_t p = (side0 ? pp : (pp >> 16)) & smask;            // P[j^1]
-                uint32_t q = Q[sb + (p ^ 1u)] & smask;
+                uint32_t p = BENES_GUARD16(side0 ? pp : (pp >> 16), smask);       // P[j^1]
+                uint32_t q = BENES_GUARD(uint32_t(Q[sb + (p ^ 1u)]), smask);
                 for (uint32_t hops = 0; hops < S; ++hops) {                // a walk claims < S/2 switches
                     j = sb + q;
                     const uint32_t t = j >> 1, side = j & 1u, g = t >> kFKappa;
@@ -221,8 +192,8 @@ k_route_fused(const uint32_t *__restrict__ P, int records, uint32_t *__restrict_
                         break;
                     }
                     pp = *reinterpret_cast<const uint32_t *>(Pcur + 2u * t);
-                    p = (side ? pp : (pp >> 16)) & smask;
-                    const uint32_t qn = Q[sb + (p ^ 1u)] & smask;
+                    p = BENES_GUARD16(side ? pp : (pp >> 16), smask);
+                    const uint32_t qn = BENES_GUARD(uint32_t(Q[sb + (p ^ 1u)]), smask);
                     const uint32_t prev = atomicCAS(reinterpret_cast<unsigned short *>(own + t),
                                                     static_cast<unsigned short>(kNone16),
                                                     static_cast<unsigned short>((uint32_t(rho) << 1) | side));
@@ -276,8 +247,8 @@ k_route_fused(const uint32_t *__restrict__ P, int records, uint32_t *__restrict_
                         const uint32_t j0 = 2u * uint32_t(t), sb = j0 & ~smask;
                         uint32_t f = j0, bk = j0, mn = j0;
                         for (uint32_t hops = 0; hops < S; ++hops) {
-                            const uint32_t pf = Pcur[f ^ 1u] & smask, pb = Pcur[bk] & smask;
-                            const uint32_t qf = Q[sb + (pf ^ 1u)] & smask, qb = Q[sb + (pb ^ 1u)] & smask;
+                            const uint32_t pf = BENES_GUARD(uint32_t(Pcur[f ^ 1u]), smask), pb = BENES_GUARD(uint32_t(Pcur[bk]), smask);
+                            const uint32_t qf = BENES_GUARD(uint32_t(Q[sb + (pf ^ 1u)]), smask), qb = BENES_GUARD(uint32_t(Q[sb + (pb ^ 1u)]), smask);
                             f = sb + qf;
                             if (f == bk) break;
                             mn = min(mn, f);
@@ -300,8 +271,8 @@ k_route_fused(const uint32_t *__restrict__ P, int records, uint32_t *__restrict_
             for (int t = tid; t < C::kPairs; t += T) {
                 const uint32_t j = 2u * t, sb = j & ~smask, jl = j & smask;
                 const uint32_t pp = *reinterpret_cast<const uint32_t *>(Pcur + j);
-                const uint32_t p0 = pp & smask, p1 = (pp >> 16) & smask;
-                const uint32_t g0 = Q[sb + (p1 ^ 1u)] & smask, g1 = Q[sb + (p0 ^ 1u)] & smask;
+                const uint32_t p0 = BENES_GUARD16(pp, smask), p1 = BENES_GUARD(pp >> 16, smask);
+                const uint32_t g0 = BENES_GUARD(uint32_t(Q[sb + (p1 ^ 1u)]), smask), g1 = BENES_GUARD(uint32_t(Q[sb + (p0 ^ 1u)]), smask);
                 *reinterpret_cast<uint32_t *>(Wd + j) = (g0 | (jl << 8)) | ((g1 | ((jl + 1u) << 8)) << 16);
             }
             __syncthreads();
@@ -344,9 +315,9 @@ k_route_fused(const uint32_t *__restrict__ P, int records, uint32_t *__restrict_
                 uint32_t sb = j & ~smask;
                 uint32_t tl = (j & smask) >> 1;
                 uint32_t c = (cw[t >> 5] >> (t & 31)) & 1u;
-                Pnext[sb + c * H + tl] = uint16_t((Pcur[j] & smask) >> 1);
-                Pnext[sb + (1u - c) * H + tl] = uint16_t((Pcur[j + 1] & smask) >> 1);
-                uint32_t q0 = Q[j] & smask;
+                Pnext[sb + c * H + tl] = uint16_t(BENES_GUARD(uint32_t(Pcur[j]), smask) >> 1);
+                Pnext[sb + (1u - c) * H + tl] = uint16_t(BENES_GUARD(uint32_t(Pcur[j + 1]), smask) >> 1);
+                uint32_t q0 = BENES_GUARD(uint32_t(Q[j]), smask);
                 uint32_t o = sb + q0;
                 cin = ((cw[o >> 6] >> ((o >> 1) & 31)) & 1u) ^ (q0 & 1u);
             }
@@ -356,6 +327,248 @@ k_route_fused(const uint32_t *__restrict__ P, int records, uint32_t *__restrict_
         __syncthreads();
         uint16_t *tmp = Pcur; Pcur = Pnext; Pnext = tmp;
     }
+}
+
+// (a block of 2^15 fills the shared memory of an SM: saying that one CTA per SM is
+// enough lets the compiler use all 64 registers a thread of a 1024-thread CTA can
+// have; left to itself it settles for 32 and spills inside the walks)
+template <int LOGM>
+__global__ void __launch_bounds__(FusedCfg<LOGM>::kThreads, (LOGM >= 15 ? 1 : 0))
+k_route_fused(const uint32_t *__restrict__ P, int records, uint32_t *__restrict__ bits, int log2n,
+              uint32_t block0) {
+    using C = FusedCfg<LOGM>;
+    constexpr int M = C::M;
+    constexpr int T = C::kThreads;
+
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    uint16_t *Pa = reinterpret_cast<uint16_t *>(smem_raw);
+    uint16_t *Q = Pa + M;
+    uint32_t *cw = reinterpret_cast<uint32_t *>(Q + M);
+    uint16_t *Pb = reinterpret_cast<uint16_t *>(cw + C::kColourWords);   // + scratch tail
+    // Pa and Pb swap roles every level, the labelling scratch always overlays
+    // the buffer P' is written to next; it starts at that buffer's first byte.
+    // Since only Pb is followed by the extra bytes, the scratch that does not
+    // fit into 2M bytes is taken from the tail behind Pb in both cases.
+    unsigned char *tail = reinterpret_cast<unsigned char *>(Pb + M);
+
+    const int tid = threadIdx.x;
+    const int n = log2n;
+    const size_t flat0 = size_t(blockIdx.x + block0) << LOGM;    // a launch may cover a range of the blocks
+    // where this CTA's words of a stage start
+    const size_t N = size_t(1) << n;
+    const size_t stage_w = N >= 64 ? N / 64 : 1;
+    const size_t perm = flat0 >> n;
+    const size_t local_first_switch = (flat0 & (N - 1)) >> 1;
+    uint32_t *my_bits = bits + perm * size_t(2 * n - 1) * stage_w + (local_first_switch >> 5);
+
+    // plain array (0), wide switch records {P[2t], P[2t+1], -, -} (1), or packed
+    // records P[2t] | P[2t+1] << LOGM | ... (2)
+    for (int j = tid; j < M; j += T) {
+        size_t f = flat0 + j;
+        uint32_t v;
+        if (records == 2) {
+            const unsigned long long w = reinterpret_cast<const unsigned long long *>(P)[f >> 1];
+            v = uint32_t(w >> ((f & 1) ? LOGM : 0));
+        } else {
+            v = records ? P[((f >> 1) << 2) | (f & 1)] : P[f];
+        }
+        Pa[j] = uint16_t(records == 2 ? (v & uint32_t(M - 1)) : BENES_GUARD(v, uint32_t(M - 1)));
+    }
+    __syncthreads();
+    fused_levels<LOGM>(Pa, Pb, Q, cw, tail, my_bits, n, n - LOGM, stage_w);
+}
+
+// ---- a block of 2^16 outputs in a thread-block cluster of two CTAs ----------------
+// The level whose sub-block spans both CTAs runs on distributed shared memory:
+// CTA r keeps outputs / inputs [r 2^15, (r+1) 2^15) of P and Q, the owners of
+// switches [r 2^14, (r+1) 2^14), the records of ruler outputs [r 2^12, (r+1) 2^12)
+// and colour words [512 r, 512 (r+1)), in the same layout the one-CTA kernel uses
+// for a block of 2^15; an index picks the CTA with its top bit.  Walkers hop
+// between the two shared memories with ordinary loads and a 16-bit
+// compare-and-swap on the owner (no multicast, no bulk copies).  The compaction
+// sends the upper half-block to CTA 0 and the lower one to CTA 1, after which
+// each CTA finishes its half exactly like the one-CTA kernel.  All values of this
+// level fit 16 bits (indices < 2^16, owner codes < 2^14, 0xFFFF = none).
+constexpr int kClusterLog2M = kFusedLog2M + 1;
+
+template <class Tp>
+struct Pair2 {                       // the same array in the two CTAs of the cluster
+    Tp *a, *b;
+    __device__ __forceinline__ Tp *of(uint32_t rank) const { return rank ? b : a; }
+};
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(FusedCfg<kFusedLog2M>::kThreads)
+k_route_cluster2(const uint32_t *__restrict__ P, int records, uint32_t *__restrict__ bits, int log2n,
+                 uint32_t block0) {
+    constexpr int LOGM = kFusedLog2M;           // per CTA
+    using C = FusedCfg<LOGM>;
+    constexpr int M = C::M;                      // outputs per CTA
+    constexpr int T = C::kThreads;
+    constexpr int R = C::kRulers;                // ruler outputs per CTA
+    constexpr int LOGR = LOGM - kFKappa;
+    constexpr uint32_t kInCta = uint32_t(M) - 1u, kSwInCta = uint32_t(M / 2) - 1u, kRInCta = uint32_t(R) - 1u;
+    constexpr uint32_t kWordsPerCta = M / 64;    // colour words per CTA
+    constexpr uint32_t kBoth = 2u * uint32_t(M) - 1u;
+    static_assert(size_t(M) + size_t(R) * 10 > size_t(2 * M), "peers live in the tail");
+
+    namespace cg = cooperative_groups;
+    cg::cluster_group cluster = cg::this_cluster();
+    const uint32_t rank = cluster.block_rank();
+
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    uint16_t *Pa = reinterpret_cast<uint16_t *>(smem_raw);
+    uint16_t *Q = Pa + M;
+    uint32_t *cw = reinterpret_cast<uint32_t *>(Q + M);
+    uint16_t *Pb = reinterpret_cast<uint16_t *>(cw + C::kColourWords);
+    unsigned char *tail = reinterpret_cast<unsigned char *>(Pb + M);
+    // scratch of the labelling, over the buffer the next level's P' goes to
+    uint16_t *own = Pb;
+    uint32_t *recm = reinterpret_cast<uint32_t *>(reinterpret_cast<unsigned char *>(Pb) + M);
+    uint32_t *list = recm + R;
+    uint16_t *peer = reinterpret_cast<uint16_t *>(tail);
+
+    const Pair2<uint16_t> Pa2{cluster.map_shared_rank(Pa, 0), cluster.map_shared_rank(Pa, 1)};
+    const Pair2<uint16_t> Q2{cluster.map_shared_rank(Q, 0), cluster.map_shared_rank(Q, 1)};
+    const Pair2<uint16_t> Pb2{cluster.map_shared_rank(Pb, 0), cluster.map_shared_rank(Pb, 1)};
+    const Pair2<uint16_t> own2{cluster.map_shared_rank(own, 0), cluster.map_shared_rank(own, 1)};
+    const Pair2<uint32_t> recm2{cluster.map_shared_rank(recm, 0), cluster.map_shared_rank(recm, 1)};
+    const Pair2<uint32_t> list2{cluster.map_shared_rank(list, 0), cluster.map_shared_rank(list, 1)};
+    const Pair2<uint32_t> cw2{cluster.map_shared_rank(cw, 0), cluster.map_shared_rank(cw, 1)};
+
+    const int tid = threadIdx.x;
+    const int lane = tid & 31;
+    const int n = log2n;
+    const int level = n - kClusterLog2M;         // recursion level of the cluster's block
+    const size_t flat0 = size_t((blockIdx.x >> 1) + block0) << kClusterLog2M;
+    const size_t N = size_t(1) << n;
+    const size_t stage_w = N / 64;
+    const size_t perm = flat0 >> n;
+    const size_t local_first_switch = (flat0 & (N - 1)) >> 1;
+    // this CTA's half of the block's words of a stage
+    uint32_t *my_bits = bits + perm * size_t(2 * n - 1) * stage_w + (local_first_switch >> 5) + rank * kWordsPerCta;
+
+    for (int j = tid; j < M; j += T) {
+        const size_t f = flat0 + rank * uint32_t(M) + j;
+        uint32_t v;
+        if (records == 2) {
+            const unsigned long long w = reinterpret_cast<const unsigned long long *>(P)[f >> 1];
+            v = uint32_t(w >> ((f & 1) ? kClusterLog2M : 0));
+        } else {
+            v = records ? P[((f >> 1) << 2) | (f & 1)] : P[f];
+        }
+        Pa[j] = uint16_t(records == 2 ? (v & kBoth) : BENES_GUARD(v, kBoth));
+    }
+    for (int t = tid; t < M / 2; t += T) own[t] = uint16_t(kNone16);
+    cluster.sync();           // both CTAs are running (and loaded) before either touches the other's memory
+    // a1: the inverse goes to the CTA that keeps that input
+    for (int j = tid; j < M; j += T) {
+        const uint32_t v = Pa[j];
+        Q2.of(v >> LOGM)[v & kInCta] = uint16_t(rank * uint32_t(M) + j);
+    }
+    cluster.sync();
+
+    // walks from this CTA's ruler outputs (its ruler switches are its own); about half of
+    // the switches and inverse entries a walker reaches are in the other CTA
+    for (int rl = tid; rl < R; rl += T) {
+        const uint32_t rho = rank * uint32_t(R) + rl;
+        const uint32_t group = rho >> 1, side0 = rho & 1u;
+        const uint32_t t0 = (group << kFKappa) | fused_slot(group, uint32_t(level));
+        uint32_t j = 2u * t0 + side0;
+        uint32_t fwd = j, part = kNone16, pr = rho ^ 1u;
+        if (!side0) own[t0 & kSwInCta] = uint16_t(rho << 1);
+        uint32_t pp = *reinterpret_cast<const uint32_t *>(Pa + 2u * (t0 & kSwInCta));
+        uint32_t p = (side0 ? pp : (pp >> 16)) & kBoth;                // P[j^1]
+        uint32_t q = Q2.of((p ^ 1u) >> LOGM)[(p ^ 1u) & kInCta];
+        for (uint32_t hops = 0; hops <= kBoth; ++hops) {                 // a walk claims < 2^15 switches
+            j = q;
+            const uint32_t t = j >> 1, side = j & 1u, g = t >> kFKappa;
+            if ((t & ((1u << kFKappa) - 1u)) == fused_slot(g, uint32_t(level))) {
+                pr = (2u * g + side) ^ 1u;                               // reached the next ruler
+                break;
+            }
+            const uint32_t c = t >> (LOGM - 1), tl = t & kSwInCta;
+            pp = *reinterpret_cast<const uint32_t *>(Pa2.of(c) + 2u * tl);
+            p = (side ? pp : (pp >> 16)) & kBoth;
+            const uint32_t qn = Q2.of((p ^ 1u) >> LOGM)[(p ^ 1u) & kInCta];
+            const uint32_t prev = atomicCAS(reinterpret_cast<unsigned short *>(own2.of(c) + tl),
+                                            static_cast<unsigned short>(kNone16),
+                                            static_cast<unsigned short>((rho << 1) | side));
+            if (prev != kNone16) {                                       // met the other walker
+                pr = prev >> 1;
+                break;
+            }
+            fwd = min(fwd, j);
+            part = min(part, j ^ 1u);
+            q = qn;
+        }
+        recm[rl] = fwd | (part << 16);
+        peer[rl] = uint16_t(pr < 2u * uint32_t(R) ? pr : rho);
+    }
+    cluster.sync();
+    // contracted list: next = peer ^ 1, minimum = own side of mine, far side of the peer's
+    for (int rl = tid; rl < R; rl += T) {
+        const uint32_t pr = peer[rl];
+        const uint32_t mn = min(recm[rl] & 0xFFFFu, recm2.of(pr >> LOGR)[pr & kRInCta] >> 16);
+        list[rl] = (pr ^ 1u) | (mn << 16);
+    }
+    cluster.sync();
+    // in-place pointer jumping; a cycle of the list has at most 2^12 words (half of the ruler outputs)
+    for (int r = 0; r < kClusterLog2M - kFKappa - 1; ++r) {
+        for (int e = tid; e < R; e += T) {
+            const uint32_t w = list[e], nx = w & 0xFFFFu;
+            const uint32_t v = list2.of((nx >> LOGR) & 1u)[nx & kRInCta];
+            const uint32_t hw = w & 0xFFFF0000u, hv = v & 0xFFFF0000u;
+            list[e] = (hw < hv ? hw : hv) | (v & 0xFFFFu);
+        }
+        cluster.sync();
+    }
+    // a4 + output side of a5 for this CTA's switches
+    for (int tl = tid; tl < M / 2; tl += T) {
+        uint32_t c;
+        const uint32_t code = own[tl];
+        if (code != kNone16) {
+            const uint32_t rr = code >> 1;
+            c = ((list2.of((rr >> LOGR) & 1u)[rr & kRInCta] >> 16) ^ code) & 1u;
+        } else {
+            // loop without ruler: walk the cycle of output 2t from both ends
+            const uint32_t j0 = 2u * (rank * uint32_t(M / 2) + tl);
+            uint32_t f = j0, bk = j0, mn = j0;
+            for (uint32_t hops = 0; hops <= kBoth; ++hops) {
+                const uint32_t pf = Pa2.of((f ^ 1u) >> LOGM)[(f ^ 1u) & kInCta], pb = Pa2.of(bk >> LOGM)[bk & kInCta];
+                const uint32_t qf = Q2.of((pf ^ 1u) >> LOGM)[(pf ^ 1u) & kInCta];
+                const uint32_t qb = Q2.of((pb ^ 1u) >> LOGM)[(pb ^ 1u) & kInCta];
+                f = qf;
+                if (f == bk) break;
+                mn = min(mn, f);
+                bk = qb ^ 1u;
+                if (bk == f) break;
+                mn = min(mn, bk);
+            }
+            c = mn & 1u;
+        }
+        const uint32_t word = __ballot_sync(0xFFFFFFFFu, c);
+        if (lane == 0) {
+            cw[tl >> 5] = word;
+            my_bits[size_t(2 * n - 2 - level) * stage_w + (tl >> 5)] = word;
+        }
+    }
+    cluster.sync();
+    // input side of a5 + a6: the upper half-block goes to CTA 0, the lower one to CTA 1
+    for (int tl = tid; tl < M / 2; tl += T) {
+        const uint32_t t = rank * uint32_t(M / 2) + tl;                  // position of the switch in either half-block
+        const uint32_t c = (cw[tl >> 5] >> (tl & 31)) & 1u;
+        const uint32_t pp = *reinterpret_cast<const uint32_t *>(Pa + 2 * tl);
+        Pb2.of(c)[t] = uint16_t((pp & 0xFFFFu) >> 1);
+        Pb2.of(c ^ 1u)[t] = uint16_t(pp >> 17);
+        const uint32_t q0 = Q[2 * tl];                                   // output fed by input 2t of the block
+        const uint32_t wq = q0 >> 6;
+        const uint32_t cin = ((cw2.of(wq / kWordsPerCta)[wq % kWordsPerCta] >> ((q0 >> 1) & 31u)) ^ q0) & 1u;
+        const uint32_t word = __ballot_sync(0xFFFFFFFFu, cin);
+        if (lane == 0) my_bits[size_t(level) * stage_w + (tl >> 5)] = word;
+    }
+    cluster.sync();
+    // from here on nothing leaves the CTA
+    fused_levels<LOGM>(Pb, Pa, Q, cw, tail, my_bits, n, level + 1, stage_w);
 }
 
 template <int LOGM>
@@ -380,14 +593,33 @@ int launch_one(const uint32_t *P, int records, size_t first_block, size_t blocks
     return launch_status();
 }
 
+int launch_cluster2(const uint32_t *P, int records, size_t first_block, size_t blocks, uint32_t *bits,
+                    int log2n, cudaStream_t s) {
+    using C = FusedCfg<kFusedLog2M>;
+    static OncePerDevice configured;
+    const int rc = configured.run([]() -> int {
+        BENES_CUDA_TRY(cudaFuncSetAttribute(k_route_cluster2, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            int(C::kSmemBytes)));
+        BENES_CUDA_TRY(cudaFuncSetAttribute(k_route_cluster2, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                            cudaSharedmemCarveoutMaxShared));
+        return BENES_OK;
+    });
+    if (rc) return rc;
+    // two CTAs per block (the cluster size is part of the kernel)
+    k_route_cluster2<<<unsigned(2 * blocks), C::kThreads, C::kSmemBytes, s>>>(P, records, bits, log2n,
+                                                                               uint32_t(first_block));
+    return launch_status();
+}
+
 }  // namespace
 
 int launch_fused(const void *Pv, int records, size_t total, int log2m, uint32_t *bits, int log2n,
                  cudaStream_t s, size_t first_block, size_t blocks) {
     const uint32_t *P = static_cast<const uint32_t *>(Pv);
-    if (log2m < 1 || log2m > kFusedLog2M) return BENES_ERR_BADARG;
+    if (log2m < 1 || log2m > kClusterLog2M) return BENES_ERR_BADARG;
     if (blocks == 0) blocks = (total >> log2m) - first_block;        // all the rest
     if (first_block + blocks > (total >> log2m)) return BENES_ERR_BADARG;
+    if (log2m == kClusterLog2M) return launch_cluster2(P, records, first_block, blocks, bits, log2n, s);
     switch (log2m) {
         case 1: return launch_one<1>(P, records, first_block, blocks, bits, log2n, s);
         case 2: return launch_one<2>(P, records, first_block, blocks, bits, log2n, s);

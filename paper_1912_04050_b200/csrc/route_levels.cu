@@ -23,6 +23,8 @@
 
 namespace cg = cooperative_groups;
 
+BENES_GUARD_TU("route_levels.cu")
+
 namespace benes {
 
 unsigned long long g_launches = 0;
@@ -62,7 +64,7 @@ k_inverse(const uint4 *__restrict__ P4, void *__restrict__ S, uint32_t *__restri
     size_t stride = size_t(gridDim.x) * blockDim.x;
     for (size_t i = size_t(blockIdx.x) * blockDim.x + threadIdx.x; i < quads; i += stride) {
         uint4 p = __ldcs(P4 + i);
-        p.x &= mmask; p.y &= mmask; p.z &= mmask; p.w &= mmask;
+        p.x = BENES_GUARD(p.x, mmask); p.y = BENES_GUARD(p.y, mmask); p.z = BENES_GUARD(p.z, mmask); p.w = BENES_GUARD(p.w, mmask);
         size_t j = i * 4;
         size_t base = j & ~size_t(mmask);
         uint32_t jl = uint32_t(j) & mmask;
@@ -123,7 +125,7 @@ k_inverse_partition(const uint32_t *__restrict__ P, void *__restrict__ S, uint2 
         // two values = one switch
         const size_t j = j0 + 2 * (size_t(i / 2) * kPartThreads + tid);
         const uint2 p = __ldcs(reinterpret_cast<const uint2 *>(P + j));
-        const uint32_t px = p.x & mmask, py = p.y & mmask;
+        const uint32_t px = BENES_GUARD(p.x, mmask), py = BENES_GUARD(p.y, mmask);
         rec_write<PACKED>(S, j >> 1, m, px, py);
         const uint32_t base = uint32_t(j) & ~mmask;
         dest[i] = base + px;
@@ -196,8 +198,8 @@ k_inverse_scatter_smem(const uint2 *__restrict__ pairs, uint32_t *__restrict__ Q
     for (int i = 0; i < kLoads; ++i) two[i] = __ldcs(src + threadIdx.x + i * 1024);
 #pragma unroll
     for (int i = 0; i < kLoads; ++i) {
-        piece[two[i].x & kInBucket] = two[i].y & mmask;
-        piece[two[i].z & kInBucket] = two[i].w & mmask;
+        piece[two[i].x & kInBucket] = BENES_GUARD(two[i].y, mmask);
+        piece[two[i].z & kInBucket] = BENES_GUARD(two[i].w, mmask);
     }
     __syncthreads();
     uint4 *dst = reinterpret_cast<uint4 *>(Q + b0);
@@ -213,7 +215,7 @@ k_inverse_scatter(const uint2 *__restrict__ pairs, uint32_t *__restrict__ Q, siz
     // the destination is forced into the bucket this pair sits in
     constexpr uint32_t kInBucket = (1u << kBucketL2Log2) - 1u;
     const size_t d = (i & ~size_t(kInBucket)) | (pr.x & kInBucket);
-    Q[d] = pr.y & mmask;
+    Q[d] = BENES_GUARD(pr.y, mmask);
 }
 
 __device__ __forceinline__ unsigned long long jump(unsigned long long w, unsigned long long t) {
@@ -246,8 +248,8 @@ k_full_label(const void *__restrict__ S, const uint32_t *__restrict__ Q,
         size_t j = 2 * t;
         size_t base = j & ~size_t(mmask);
         uint32_t b32 = uint32_t(base);
-        uint32_t g0 = b32 + (__ldg(Q + base + (p1 ^ 1u)) & mmask);
-        uint32_t g1 = b32 + (__ldg(Q + base + (p0 ^ 1u)) & mmask);
+        uint32_t g0 = b32 + BENES_GUARD(__ldg(Q + base + (p1 ^ 1u)), mmask);
+        uint32_t g1 = b32 + BENES_GUARD(__ldg(Q + base + (p0 ^ 1u)), mmask);
         ulonglong2 a;
         a.x = make_word(g0, uint32_t(j));
         a.y = make_word(g1, uint32_t(j) + 1u);
@@ -325,7 +327,7 @@ k_split(const void *__restrict__ S, const uint4 *__restrict__ Q4, void *__restri
             rec_write<NEXT_PACKED>(Sn, r, m - 1, (c0 ? py0 : px0) >> 1, (c1 ? py1 : px1) >> 1);
             rec_write<NEXT_PACKED>(Sn, r + (H >> 1), m - 1, (c0 ? px0 : py0) >> 1, (c1 ? px1 : py1) >> 1);
         }
-        q.x &= mmask; q.y &= mmask; q.z &= mmask; q.w &= mmask;
+        q.x = BENES_GUARD(q.x, mmask); q.y = BENES_GUARD(q.y, mmask); q.z = BENES_GUARD(q.z, mmask); q.w = BENES_GUARD(q.w, mmask);
         // colour of the output fed by input 2t (2t+2): that output's switch bit, flipped for an odd output
         const uint32_t cin0 = ((colours[q.x >> 6] >> ((q.x >> 1) & 31u)) ^ q.x) & 1u;
         const uint32_t cin1 = ((colours[q.z >> 6] >> ((q.z >> 1) & 31u)) ^ q.z) & 1u;

@@ -36,6 +36,8 @@
 // level.  So the result never depends on the sampling.
 #include "common.cuh"
 
+BENES_GUARD_TU("route_sampled.cu")
+
 namespace benes {
 
 
@@ -98,9 +100,9 @@ k_walk(void *__restrict__ Sv, const uint32_t *__restrict__ Q, uint4 *__restrict_
     } else {
         const uint4 r = __ldcg(S16 + t0);
         if (!side0) reinterpret_cast<uint32_t *>(S16 + t0)[2] = rho << 1;
-        p = (side0 ? r.x : r.y) & mmask;
+        p = BENES_GUARD(side0 ? r.x : r.y, mmask);
     }
-    uint32_t q = __ldcg(Q + base + (p ^ 1u)) & mmask;
+    uint32_t q = BENES_GUARD(__ldcg(Q + base + (p ^ 1u)), mmask);
     for (;;) {
         j = base + q;
         const uint32_t t = j >> 1, side = j & 1u, g = t >> kappa;
@@ -120,7 +122,7 @@ k_walk(void *__restrict__ Sv, const uint32_t *__restrict__ Q, uint4 *__restrict_
             const unsigned long long w = atomicAnd(S8 + t, mine | low_ones);
             p = uint32_t(w >> (side ? 0 : m)) & mmask;
             // next hop's gather, issued before the claim is looked at (harmless if we stop)
-            qn = __ldcg(Q + base + (p ^ 1u)) & mmask;
+            qn = BENES_GUARD(__ldcg(Q + base + (p ^ 1u)), mmask);
             const uint32_t prev = uint32_t(w >> cshift);
             met = prev != none8;
             if (met) {
@@ -129,8 +131,8 @@ k_walk(void *__restrict__ Sv, const uint32_t *__restrict__ Q, uint4 *__restrict_
             }
         } else {
             const uint4 r = __ldcg(S16 + t);
-            p = (side ? r.x : r.y) & mmask;
-            qn = __ldcg(Q + base + (p ^ 1u)) & mmask;
+            p = BENES_GUARD(side ? r.x : r.y, mmask);
+            qn = BENES_GUARD(__ldcg(Q + base + (p ^ 1u)), mmask);
             uint32_t prev = r.z;
             if (prev == kUnowned)
                 prev = atomicCAS(reinterpret_cast<uint32_t *>(S16 + t) + 2, kUnowned, (rho << 1) | side);
@@ -151,7 +153,7 @@ k_combine(const uint4 *__restrict__ rec, unsigned long long *__restrict__ W, uin
     const uint32_t rho = blockIdx.x * kThreads + threadIdx.x;
     if (rho >= rulers) return;
     const uint4 a = rec[rho];
-    const uint32_t peer = a.z < rulers ? a.z : rho;
+    const uint32_t peer = BENES_GUARD_BELOW(a.z, rulers, rho);
     const uint4 b = __ldg(rec + peer);
     W[rho] = make_word(peer ^ 1u, min(a.x, b.y));
 }
@@ -183,7 +185,7 @@ k_list_walk_pairs(const ulonglong2 *__restrict__ W2p, uint32_t *__restrict__ own
     uint32_t fwd = uint32_t(own >> 32), part = kUnowned, peer = sigma ^ 1u, hops = 0;
     for (;;) {
         // (a batch need not be a power of two: an index a raised gate left undefined is clamped, not masked)
-        const uint32_t e = uint32_t(own), q = (e >> 1) < pairs ? (e >> 1) : 0u, side = e & 1u, g = q >> kPairGroupLog2;
+        const uint32_t e = uint32_t(own), q = BENES_GUARD_BELOW(e >> 1, pairs, 0u), side = e & 1u, g = q >> kPairGroupLog2;
         if ((q & kmask) == ruler_slot(g, salt, kmask)) {           // reached the next ruler pair
             peer = (2u * g + side) ^ 1u;
             break;
@@ -220,7 +222,7 @@ k_list_walk_pairs(const ulonglong2 *__restrict__ W2p, uint32_t *__restrict__ own
 __device__ __forceinline__ uint32_t list_cycle_min(const unsigned long long *W, uint32_t e0, uint32_t words,
                                                    uint32_t cap, uint32_t *gate) {
     unsigned long long v = __ldcg(W + e0);
-    uint32_t mn = uint32_t(v >> 32), e = uint32_t(v) < words ? uint32_t(v) : 0u, hops = 0;
+    uint32_t mn = uint32_t(v >> 32), e = BENES_GUARD_BELOW(uint32_t(v), words, 0u), hops = 0;
     while (e != e0) {
         if (++hops > cap) {
             *gate = 1u;
@@ -228,7 +230,7 @@ __device__ __forceinline__ uint32_t list_cycle_min(const unsigned long long *W, 
         }
         v = __ldcg(W + e);
         mn = min(mn, uint32_t(v >> 32));       // words rewritten meanwhile hold the minimum of this same cycle
-        e = uint32_t(v) < words ? uint32_t(v) : 0u;
+        e = BENES_GUARD_BELOW(uint32_t(v), words, 0u);
     }
     return mn;
 }
@@ -407,8 +409,8 @@ __device__ __forceinline__ uint32_t loop_colour(const void *S, const uint32_t *Q
     uint32_t pf = p_odd;                 // P[f ^ 1]
     uint32_t pb = p_even;                // P[bk]
     for (;;) {
-        const uint32_t qf = __ldg(Q + base + (pf ^ 1u)) & mmask;        // g(f)
-        const uint32_t qb = __ldg(Q + base + (pb ^ 1u)) & mmask;        // g(bk ^ 1)
+        const uint32_t qf = BENES_GUARD(__ldg(Q + base + (pf ^ 1u)), mmask);        // g(f)
+        const uint32_t qb = BENES_GUARD(__ldg(Q + base + (pb ^ 1u)), mmask);        // g(bk ^ 1)
         f = base + qf;
         if (f == bk) break;                                             // forwards reached the part walked backwards
         mn = min(mn, f);
@@ -428,7 +430,7 @@ __device__ __forceinline__ uint32_t loop_colour(const void *S, const uint32_t *Q
 
 // colour of output 2t from the owner of switch t
 __device__ __forceinline__ uint32_t owner_colour(const uint32_t *cb, uint32_t code, uint32_t rulers) {
-    const uint32_t rho = (code >> 1) < rulers ? code >> 1 : 0u;
+    const uint32_t rho = BENES_GUARD_BELOW(code >> 1, rulers, 0u);
     return ((__ldg(cb + (rho >> 5)) >> (rho & 31u)) ^ code) & 1u;
 }
 
@@ -488,8 +490,8 @@ k_colour(const void *__restrict__ S, const uint32_t *__restrict__ Q,
             own0 = l0 != none; own1 = l1 != none;
             code0 = rb + l0; code1 = rb + l1;                    // owner local to the block -> global
         } else {
-            px0 = r0.x & mmask; py0 = r0.y & mmask; code0 = r0.z; own0 = code0 != none;
-            px1 = r1.x & mmask; py1 = r1.y & mmask; code1 = r1.z; own1 = code1 != none;
+            px0 = BENES_GUARD(r0.x, mmask); py0 = BENES_GUARD(r0.y, mmask); code0 = r0.z; own0 = code0 != none;
+            px1 = BENES_GUARD(r1.x, mmask); py1 = BENES_GUARD(r1.y, mmask); code1 = r1.z; own1 = code1 != none;
         }
         // all but the switches of loops without ruler are owned
         const uint32_t c0 = own0 ? owner_colour(cb, code0, rulers)

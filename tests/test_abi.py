@@ -33,6 +33,15 @@ def test_header_symbols_are_exported_and_bound(lib):
     assert sorted(binding.SYMBOLS) == names
 
 
+def test_checked_build_has_the_same_abi():
+    path = build.build(debug=True)
+    raw = ctypes.CDLL(path)
+    for name in _declared():
+        assert hasattr(raw, name), name
+    assert raw.benes_debug_build() == 1
+    assert ctypes.CDLL(binding.LIB_PATH).benes_debug_build() == 0
+
+
 def test_sizing_helpers(lib):
     assert lib.benes_switch_words(10, 1) == 19 * 16
     assert lib.benes_switch_words(8, 16384) == 16384 * 15 * 4

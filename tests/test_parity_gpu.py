@@ -108,6 +108,28 @@ def test_route_every_ruler_spacing(kappa, labelling_options):
     assert np.array_equal(gpu_route(perm, 16), oracle.route(perm, 16))
 
 
+@pytest.fixture
+def cluster_mode():
+    c0 = binding.benes_get_option(binding.OPT_CLUSTER)
+    binding.benes_set_option(binding.OPT_CLUSTER, 1)
+    yield
+    binding.benes_set_option(binding.OPT_CLUSTER, c0)
+
+
+@pytest.mark.parametrize("n,batch", [(16, 1), (16, 3), (16, 64), (17, 1), (17, 3), (17, 64), (18, 5), (20, 1), (22, 1)])
+def test_route_blocks_of_2p16_in_clusters_of_two_ctas(n, batch, cluster_mode):
+    """Whole permutations of 2^16 (one cluster each) and the tails of larger ones."""
+    perm = inputs.random_perm_batch(n, batch, seed0=500 + n + batch)
+    assert np.array_equal(gpu_route(perm, n), oracle.route(perm, n))
+
+
+@pytest.mark.parametrize("n", [16, 17, 19])
+@pytest.mark.parametrize("kind", ["identity", "shift1", "bitrev", "transpose", "sattolo"])
+def test_route_structured_in_clusters(n, kind, cluster_mode):
+    perm = inputs.structured_perms(n)[kind]
+    assert np.array_equal(gpu_route(perm, n), oracle.route(perm, n))
+
+
 @pytest.mark.parametrize("cap", [1, 3, 40])
 def test_route_walks_that_give_up_fall_back_to_full_pointer_jumping(cap, labelling_options):
     """With a tiny hop limit almost every level raises its gate and is relabelled
