@@ -87,6 +87,11 @@ KIND_SOURCE = {"walk": "route_sampled.cu", "colour": "route_sampled.cu", "fused"
                "split": "route_levels.cu", "inverse": "route_levels.cu", "apply_fused": "apply_fused.cu"}
 
 
+def binding_packed_level0(n: int, kappa: int) -> bool:
+    """Whether level 0 of a permutation of 2^n uses packed 8-byte records (the library's rule)."""
+    return kappa != 0 and 3 * n - kappa + 1 < 64
+
+
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -455,25 +460,40 @@ def time_steps(case: GpuCase, steps: int, flush):
     return [a.elapsed_time(b) for a, b in pairs]
 
 
-def probe_gather(binding, table, stream):
-    """Independent random 4-byte gathers from `table` (a power-of-two number of words): G/s."""
+PROBE_MODES = {
+    # name: (mode, record bytes, records = elements >> shift, what it stands for)
+    "load4": (0, 4, 0, "4-byte load from an array of one word per element (the inverse entry of a hop)"),
+    "load16": (1, 16, 1, "16-byte load of a wide switch record"),
+    "load16_cas": (2, 16, 1, "16-byte load + compare-and-swap on its owner word (a visit of a wide record)"),
+    "and64": (3, 8, 1, "64-bit atomic AND on an 8-byte record (a visit of a packed record)"),
+    "store4": (4, 16, 1, "4-byte store into a 16-byte record"),
+}
+
+
+def probe_random_access(binding, stream, log2_elems: int):
+    """Independent random accesses, one per switch of a level of 2^log2_elems outputs, on
+    arrays of that level's sizes: G operations/s per access pattern (best of 3)."""
     import torch
-    words = table.numel()
-    log2w = words.bit_length() - 1
+    switches = 1 << (log2_elems - 1)
+    table = torch.empty(switches * 16, dtype=torch.uint8, device="cuda")
     sink = torch.zeros(1, dtype=torch.int32, device="cuda")
-    gathers = min(1 << 28, max(1 << 24, 4 * words))
-    best = None
-    for i in range(6):
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        binding.benes_probe_gather(table, log2w, gathers, sink, stream)
-        e1.record(stream)
-        torch.cuda.synchronize()
-        if i >= 2:
+    out = {}
+    for name, (mode, rbytes, shift, what) in PROBE_MODES.items():
+        best = None
+        for _ in range(3):
+            table.fill_(255)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record(stream)
+            binding.benes_probe_random_access(table, log2_elems - shift, rbytes, mode, switches, sink, stream)
+            e1.record(stream)
+            torch.cuda.synchronize()
             ms = e0.elapsed_time(e1)
             best = ms if best is None else min(best, ms)
-    return {"value": gathers / (best * 1e-3) / 1e9, "unit": "G gathers/s", "gathers": gathers,
-            "table_bytes": words * 4, "ms": best}
+        out[name] = {"g_ops_per_s": switches / (best * 1e-3) / 1e9, "ms": best, "ops": switches,
+                     "table_bytes": (1 << (log2_elems - shift)) * rbytes, "what": what}
+    del table
+    return out
 
 
 def side_workload(name: str, rank: int, stream, flush, steps: int = 10):
@@ -520,9 +540,17 @@ def run_gpu(args):
 
     if args.cluster is not None:
         binding.benes_set_option(binding.OPT_CLUSTER, args.cluster)
+    if args.apply_fused is not None:
+        binding.benes_set_option(binding.OPT_APPLY_FUSED, args.apply_fused)
 
     name = args.workload
     stream = torch.cuda.Stream()
+    if args.probe_only:
+        n0, b0 = WORKLOADS[name][0], WORKLOADS[name][1]
+        with torch.cuda.stream(stream):
+            print(json.dumps({"random_access_probe": probe_random_access(binding, stream, n0 + (b0.bit_length() - 1))}),
+                  flush=True)
+        return
     case = GpuCase(name, rank, stream)
     n, batch, ebytes, elems = case.n, case.batch, case.ebytes, case.elems
     flush = None if case.input_bytes > L2_BYTES else L2Flush()
@@ -599,9 +627,9 @@ def run_gpu(args):
         assert torch.equal(out_p, case.d_out.cpu()), "end-to-end payload differs from the device-resident run"
         del perm_p, x_p, out_p
 
-        gather = None
-        if rank == 0 and (case.d_perm.numel() & (case.d_perm.numel() - 1)) == 0 and case.d_perm.numel() >= 1 << 20:
-            gather = probe_gather(binding, case.d_perm, stream)
+        probe = None
+        if rank == 0 and n >= 20 and not args.no_probe:
+            probe = probe_random_access(binding, stream, n + (batch.bit_length() - 1))
 
     ms_step = sum(step_ms) / len(step_ms)
     ms_step, e2e_ms, route_ms, apply_ms = max_over_ranks([ms_step, e2e_ms, route_ms, apply_ms], dist, "cuda")
@@ -624,24 +652,24 @@ def run_gpu(args):
                 "algorithmic_bytes_per_launch": bpe * elems,
                 "avg_launch_ms": per_launch_s * 1e3, "launches_timed": dom["launches"],
             }
-            if top == "walk" and per_level.get("walk") and gather:
-                # the walk is a chain of dependent random accesses: per switch one record and
-                # one 4-byte inverse entry (the claim hits the record's sector), i.e. one access
-                # per element.  Level 0 is the launch whose block is furthest above the L2, so
-                # its accesses all go to DRAM; the ceiling is the rate of independent random
-                # gathers from the same-sized array, measured in this run.
-                acc = float(elems) / (per_level["walk"][0] * 1e-3) / 1e9
+            traffic = roofline["traffic"]
+            if traffic:
+                # what the DRAM actually moved for this kernel (ncu counters of the same workload)
+                roofline["dram_gbs"] = traffic / per_launch_s / 1e9
+                roofline["dram_frac"] = traffic / per_launch_s / 1e9 / peak
+            if top == "walk" and per_level.get("walk") and probe:
+                # The walk is a chain of dependent random accesses: per switch one record visit
+                # (load + claim) and one 4-byte inverse entry.  Level 0 is the launch whose block
+                # is furthest above the L2.  The time the same accesses take when they are
+                # independent (measured in this run on arrays of the same sizes) is the floor.
+                visit = "load16_cas" if per_level["walk"][0] and not binding_packed_level0(n, kappa) else "and64"
+                floor_ms = probe[visit]["ms"] + probe["load4"]["ms"]
                 roofline["random_access"] = {
                     "launch": "level 0", "ms": per_level["walk"][0],
-                    "achieved": acc, "unit": "G accesses/s", "peak": gather["value"],
-                    "peak_source": "this run: %d independent random 4-byte gathers from the %d MiB "
-                                   "permutation array (benes_probe_gather), best of 4"
-                                   % (gather["gathers"], gather["table_bytes"] >> 20),
-                    "frac": acc / gather["value"],
-                    # the claim (an atomic on the record) counted as a third memory operation
-                    # per switch, i.e. 1.5 per element
-                    "achieved_with_claims": 1.5 * acc,
-                    "frac_with_claims": 1.5 * acc / gather["value"]}
+                    "floor_ms": floor_ms, "frac": floor_ms / per_level["walk"][0],
+                    "floor": "independent accesses of the same kinds and counts on arrays of the same "
+                             "sizes (benes_probe_random_access, this run): %s %.3f ms + load4 %.3f ms"
+                             % (visit, probe[visit]["ms"], probe["load4"]["ms"])}
         bits_bytes = case.d_bits.numel() * 4
         line = {
             "metric": METRIC, "value": whole_job_value(elems, world, ms_step), "unit": UNIT,
@@ -669,8 +697,8 @@ def run_gpu(args):
                                                      if k in ("walk", "colour", "split", "list_label", "list_walk")},
                           "kernel_launches_per_step": {k: v["launches"] // args.steps for k, v in kinds.items()}},
         }
-        if gather:
-            line["gather_probe"] = gather
+        if probe:
+            line["random_access_probe"] = probe
         if world == 1 and name == "c4" and not args.no_side_workloads:
             del case
             torch.cuda.empty_cache()
@@ -693,10 +721,15 @@ def main():
     ap.add_argument("--workload", default="c4", choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-side-workloads", action="store_true")
+    ap.add_argument("--no-probe", action="store_true", help="skip the random-access probe")
+    ap.add_argument("--probe-only", action="store_true",
+                    help="run only the random-access probe for the workload's size (for profiling it)")
     ap.add_argument("--kappa", type=int, default=None,
                     help="ruler spacing (log2) of the loop labelling; 0 = full pointer jumping")
     ap.add_argument("--cluster", type=int, default=None,
                     help="1: blocks of 2^16 finished by clusters of two CTAs; 0: blocks of 2^15 in one CTA")
+    ap.add_argument("--apply-fused", type=int, default=None,
+                    help="0: one payload-apply kernel per stage; 1: several stages per pass (default)")
     ap.add_argument("--rank-check", action="store_true",
                     help="run only the rank plumbing on the CPU (gloo); used by the tests")
     args = ap.parse_args()

@@ -257,15 +257,20 @@ const char *benes_profile_kind_name(int kind);
 int benes_shard_batch(int batch, int world, int rank, int *first, int *count);
 
 /*
- * Measurement aid (no step of the method): `gathers` (<= 2^32) independent random
- * 4-byte reads from table[0 .. 2^log2_words), eight in flight per thread,
- * enqueued on `stream`; the caller times it with events.  The ruler walks are
- * chains of random accesses, and this is the rate they are compared with.
- * `sink` is one device word; it is written only if the words a thread read
+ * Measurement aid (no step of the method): `ops` (<= 2^32) random accesses to
+ * table[0 .. 2^log2_records * record_bytes), each to a different pseudo-randomly
+ * placed record when ops <= 2^log2_records, two in flight per thread, enqueued on
+ * `stream`; the caller times it with events.  The ruler walks are chains of such
+ * accesses, and these are the rates (and, under a profiler, the DRAM bytes per
+ * access) they are compared with.  mode 0: 4-byte load; 1: 16-byte load; 2:
+ * 16-byte load, then compare-and-swap on the record's third word; 3: 64-bit atomic
+ * AND on the record's first 8 bytes; 4: 4-byte store to the third word.  Modes 2-4
+ * overwrite the table.  record_bytes: a multiple of 4 / 16 / 16 / 8 / 16 for modes
+ * 0..4.  `sink` is one device word; it is written only if the words a thread read
  * xor to one particular value (so that the reads cannot be dropped).
  */
-int benes_probe_gather(const uint32_t *table, int log2_words, size_t gathers, uint32_t *sink,
-                       benes_stream_t stream);
+int benes_probe_random_access(void *table, int log2_records, int record_bytes, int mode, size_t ops,
+                              uint32_t *sink, benes_stream_t stream);
 
 /*
  * Checked build.  Every index a kernel forms from data is forced into range (a

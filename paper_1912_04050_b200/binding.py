@@ -53,7 +53,7 @@ SYMBOLS = {
                                 ctypes.POINTER(ctypes.c_double)]),
     "benes_profile_kind_name": (ctypes.c_char_p, [_i]),
     "benes_shard_batch": (_i, [_i, _i, _i, ctypes.POINTER(_i), ctypes.POINTER(_i)]),
-    "benes_probe_gather": (_i, [_vp, _i, _sz, _vp, _vp]),
+    "benes_probe_random_access": (_i, [_vp, _i, _i, _i, _sz, _vp, _vp]),
     "benes_debug_build": (_i, []),
     "benes_debug_guard_hits": (_i, [ctypes.POINTER(ctypes.c_ulonglong), ctypes.c_char_p, _sz, _i]),
     "benes_fused_log2m": (_i, []),
@@ -284,9 +284,10 @@ def benes_shard_batch(batch: int, world: int, rank: int):
     return first.value, count.value
 
 
-def benes_probe_gather(table: torch.Tensor, log2_words: int, gathers: int, sink: torch.Tensor, stream=None) -> None:
-    _check(load().benes_probe_gather(_dev_ptr(table, "table"), log2_words, gathers, _dev_ptr(sink, "sink"),
-                                     _stream(stream)), "benes_probe_gather")
+def benes_probe_random_access(table: torch.Tensor, log2_records: int, record_bytes: int, mode: int, ops: int,
+                              sink: torch.Tensor, stream=None) -> None:
+    _check(load().benes_probe_random_access(_dev_ptr(table, "table"), log2_records, record_bytes, mode, ops,
+                                            _dev_ptr(sink, "sink"), _stream(stream)), "benes_probe_random_access")
 
 
 def benes_debug_build() -> bool:
