@@ -132,12 +132,17 @@ int benes_export_butterfly(const uint32_t *switch_bits, uint32_t *butterfly_bits
  * batch * N * elem_bytes must not exceed BENES_STATIC_SCRATCH_BYTES, otherwise
  * BENES_ERR_TOO_LARGE is returned and nothing is enqueued.
  *
- * The first call on each device looks up the array's device address (a
- * runtime query, no allocation); make that first call outside any stream
- * capture.  All calls share the one array and it keeps the previous call's
- * contents (nothing needs clearing: each stage overwrites all it later
- * reads).  Two calls whose kernels can overlap on the GPU (different streams,
- * no ordering) race on it: keep them on one stream or order them yourself.
+ * The first call on each device looks up the array's device address with the
+ * runtime.  That query allocates nothing by itself, but it can be the moment
+ * the CUDA runtime loads the part of the library that holds the array and
+ * reserves its 4 MiB on that device.  So make one call per device at start-up:
+ * before the rest of the device memory is handed to another allocator (a
+ * process that has already given everything away can see BENES_ERR_CUDA from
+ * this first call), and outside any stream capture.  All calls share the one
+ * array and it keeps the previous call's contents (nothing needs clearing:
+ * each stage overwrites all it later reads).  Two calls whose kernels can
+ * overlap on the GPU (different streams, no ordering) race on it: keep them on
+ * one stream or order them yourself.
  */
 #define BENES_STATIC_SCRATCH_BYTES (4u << 20)
 int benes_apply_static(const uint32_t *switch_bits, const void *in, void *out, int elem_bytes,

@@ -253,6 +253,15 @@ def test_config4_n2p26_u64_payload():
     assert np.array_equal(bits, oracle.route(perm, n))
 
 
+def test_route_n2p27_matches_the_oracle():
+    """One size above the headline, word for word (the oracle needs about two minutes)."""
+    n = 27
+    perm = inputs.random_perm(n, 7)
+    bits = gpu_route(perm, n)
+    assert np.array_equal(bits, oracle.route(perm, n))
+    binding.benes_release_workspace()
+
+
 @pytest.mark.parametrize("n_elems,batch", [(1, 2), (3, 4), (5, 3), (100, 5), (1000, 2), (4097, 3),
                                            (40000, 2), (100000, 1), (300001, 1)])
 def test_sizes_that_are_not_a_power_of_two(n_elems, batch):

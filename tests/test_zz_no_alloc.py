@@ -61,3 +61,34 @@ def test_static_apply_refuses_what_does_not_fit():
         binding.benes_apply_static(dummy, dummy, torch.zeros_like(dummy), 4, 10, 1 + (1 << 10))
     assert e.value.status == binding.BENES_ERR_TOO_LARGE
     assert "scratch" in binding.status_string(binding.BENES_ERR_TOO_LARGE)
+
+
+def test_static_apply_needs_no_workspace_and_no_device_memory():
+    """What the entry point is for: with a caller workspace of 256 bytes installed, any
+    internal request for scratch fails (the regular entry point does, below), yet the
+    allocation-free one still works, and the free device memory is the same before and
+    after the call."""
+    n, batch = 17, 2
+    perm = inputs.random_perm_batch(n, batch, seed0=77)
+    x = inputs.payload_u64(batch << n, 5).reshape(batch, -1)
+    d_x = _dev(x)
+    bits = binding.route(_dev(perm))
+    got = torch.empty_like(d_x)
+    binding.benes_apply_static(bits, d_x, got, 8, n, batch)          # first call on this device: address look-up
+    torch.cuda.synchronize()
+    tiny = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    binding.benes_set_workspace(tiny)
+    try:
+        with pytest.raises(binding.BenesError) as e:
+            binding.benes_apply_ex(bits, d_x, torch.empty_like(d_x), 8, n, batch)
+        assert e.value.status == binding.BENES_ERR_NOMEM
+        got.fill_(-1)
+        torch.cuda.synchronize()
+        free0, _ = torch.cuda.mem_get_info()
+        binding.benes_apply_static(bits, d_x, got, 8, n, batch)
+        torch.cuda.synchronize()
+        free1, _ = torch.cuda.mem_get_info()
+        assert free1 == free0
+    finally:
+        binding.benes_set_workspace(None)
+    assert np.array_equal(got.cpu().numpy().view(np.uint64), np.take_along_axis(x, perm.astype(np.int64), axis=1))
