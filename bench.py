@@ -53,8 +53,9 @@ WORKLOADS = {
 }
 STRUCTURED = {"c5i": "identity", "c5h": "shift1", "c5b": "bitrev", "c5t": "transpose"}
 L2_BYTES = 126 << 20
-# workloads whose summary rides along in the default (C4) line
-SIDE_WORKLOADS = ("c3", "c2")
+# workloads whose summary rides along in the default (C4) line: the rest of the metric's range (C3,
+# C2) and the remaining configurations (C1, the five structured permutations of C5)
+SIDE_WORKLOADS = ("c3", "c2", "c1", "c5s", "c5i", "c5h", "c5b", "c5t")
 
 
 def algorithmic_bytes_per_element(kind: str, ebytes: int, kappa: int) -> float:
@@ -515,8 +516,11 @@ def side_workload(name: str, rank: int, stream, flush, steps: int = 10):
         r2.record(stream)
         torch.cuda.synchronize()
     med = statistics.median(ms)
-    return {"workload": case.desc, "ms_per_step": med, "best_ms": min(ms), "steps": steps,
-            "value": case.elems / (med * 1e-3), "unit": UNIT, "l2": "flushed between steps",
+    del case
+    torch.cuda.empty_cache()
+    return {"workload": WORKLOADS[name][4], "ms_per_step": med, "best_ms": min(ms), "steps": steps,
+            "value": (WORKLOADS[name][1] << WORKLOADS[name][0]) / (med * 1e-3), "unit": UNIT,
+            "l2": "flushed between steps",
             "route_ms": r0.elapsed_time(r1), "apply_ms": r1.elapsed_time(r2)}
 
 

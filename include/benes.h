@@ -212,6 +212,10 @@ int benes_validate_perm(const uint32_t *perm, int log2n, int batch, benes_stream
  *       and the tail of larger ones) are finished by a thread-block cluster of two
  *       CTAs over distributed shared memory instead of one more level in global
  *       memory; 0 = blocks of 2^15 in one CTA.  Same result.
+ *   BENES_OPT_WALK_PAIRS : at levels with packed 8-byte records a thread can advance the
+ *       two walks that leave one ruler switch together (their chains of dependent
+ *       accesses overlap).  0 = never, 1 (default) = where the halved number of
+ *       threads still fills the GPU, 2 = at every such level.  Same result.
  * benes_set_option returns BENES_OK or BENES_ERR_BADARG; benes_get_option
  * returns the value, or BENES_ERR_BADARG for an unknown key.
  */
@@ -221,6 +225,7 @@ int benes_validate_perm(const uint32_t *perm, int log2n, int batch, benes_stream
 #define BENES_OPT_INVERSE_PARTITIONED 3
 #define BENES_OPT_CHUNK_LOG2 4
 #define BENES_OPT_CLUSTER 5
+#define BENES_OPT_WALK_PAIRS 6
 int benes_set_option(int key, int value);
 int benes_get_option(int key);
 

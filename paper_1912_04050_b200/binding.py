@@ -234,6 +234,7 @@ OPT_APPLY_FUSED = 2
 OPT_INVERSE_PARTITIONED = 3
 OPT_CHUNK_LOG2 = 4
 OPT_CLUSTER = 5
+OPT_WALK_PAIRS = 6
 
 
 def benes_set_option(key: int, value: int) -> None:

@@ -45,6 +45,7 @@ struct Options {
     int inverse_partitioned = 1;
     int chunk_log2 = 30;            // flat elements processed together by the per-level path (indices are 32 bit)
     int cluster = 0;                // 1: blocks of 2^16 are finished by clusters of two CTAs
+    int walk_pairs = 1;             // two ruler walks per thread: 0 never, 1 where it pays, 2 wherever possible
 };
 Options g_opt;
 constexpr int kMaxLevels = 32;
@@ -210,8 +211,8 @@ int route_levels(const uint32_t *perm, int n, size_t batch, uint32_t *bits, char
         if (kappa) {
             // ruler-sampled labelling; raises `gate` if a walk had to give up
             gate = gates + level;
-            if ((rc = sampled_label(S, pk, Q, Sbuf[cur ^ 1], pk_next, sc, T, m, kappa, uint32_t(level), cap, L,
-                                    out_stage, gate, s)))
+            if ((rc = sampled_label(S, pk, Q, Sbuf[cur ^ 1], pk_next, sc, T, m, kappa, uint32_t(level), cap,
+                                    opt.walk_pairs, L, out_stage, gate, s)))
                 return rc;
         }
         // pointer jumping over all outputs: the whole labelling when sampling is
@@ -632,6 +633,10 @@ int benes_set_option(int key, int value) {
             if (value != 0 && value != 1) return BENES_ERR_BADARG;
             g_opt.cluster = value;
             return BENES_OK;
+        case BENES_OPT_WALK_PAIRS:
+            if (value < 0 || value > 2) return BENES_ERR_BADARG;
+            g_opt.walk_pairs = value;
+            return BENES_OK;
         default: return BENES_ERR_BADARG;
     }
 }
@@ -645,6 +650,7 @@ int benes_get_option(int key) {
         case BENES_OPT_INVERSE_PARTITIONED: return g_opt.inverse_partitioned;
         case BENES_OPT_CHUNK_LOG2: return g_opt.chunk_log2;
         case BENES_OPT_CLUSTER: return g_opt.cluster;
+        case BENES_OPT_WALK_PAIRS: return g_opt.walk_pairs;
         default: return BENES_ERR_BADARG;
     }
 }

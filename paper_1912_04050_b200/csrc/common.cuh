@@ -278,8 +278,8 @@ void sampled_scratch_carve(char *base, size_t total, int kappa, SampledScratch *
 // level's records Sn; raises *gate if some walk exceeded `cap` hops (the level
 // must then be relabelled and Sn rewritten).
 int sampled_label(void *S, bool packed, const uint32_t *Q, void *Sn, bool next_packed,
-                  const SampledScratch &sc, size_t total, int log2m, int kappa, uint32_t salt, uint32_t cap, BitsLayout L, int out_stage,
-                  uint32_t *gate, cudaStream_t s);
+                  const SampledScratch &sc, size_t total, int log2m, int kappa, uint32_t salt, uint32_t cap,
+                  int walk_pairs, BitsLayout L, int out_stage, uint32_t *gate, cudaStream_t s);
 // owner[0] and owner[1] must be all kUnowned before the first sampled_label.
 int sampled_scratch_reset(const SampledScratch &sc, size_t total, int kappa, cudaStream_t s);
 

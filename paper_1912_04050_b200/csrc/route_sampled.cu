@@ -147,6 +147,90 @@ k_walk(void *__restrict__ Sv, const uint32_t *__restrict__ Q, uint4 *__restrict_
     rec[rho] = make_uint4(fwd, part, peer, 0u);
 }
 
+// Step 2, packed records, 2 G walkers per thread: the two ruler outputs of each of G
+// neighbouring ruler switches (the two walks of a switch leave it in opposite
+// directions).  A hop is a chain of two dependent L2 accesses and most lanes of a
+// warp are idle while its longest walk lasts; advancing a thread's walks together,
+// one hop each per round, overlaps their chains.  Same claims and records as
+// k_walk<true>.  The hop limit counts rounds.
+template <int G>
+__global__ void __launch_bounds__(kWalkThreads)
+k_walk_multi(unsigned long long *__restrict__ S8, const uint32_t *__restrict__ Q, uint4 *__restrict__ rec,
+             uint32_t groups, int m, int kappa, uint32_t salt, uint32_t cap, uint32_t *__restrict__ gate) {
+    constexpr int W = 2 * G;
+    const uint32_t group0 = (blockIdx.x * kWalkThreads + threadIdx.x) * G;     // groups is a multiple of G
+    if (group0 >= groups) return;
+    const uint32_t mmask = (1u << m) - 1u;
+    const uint32_t kmask = (1u << kappa) - 1u;
+    const int cshift = 2 * m;
+    const unsigned long long low_ones = (1ull << cshift) - 1ull;
+    const uint32_t none8 = uint32_t(~0ull >> cshift);
+    const uint32_t rho0 = 2u * group0;                               // walker i is ruler output rho0 + i
+    // G neighbouring groups lie in one block (a block has at least 2^7 ruler outputs)
+    const uint32_t base = (2u * (group0 << kappa)) & ~mmask;
+    const uint32_t rho_base = base >> kappa;
+    uint32_t q[W], fwd[W], part[W], peer[W];
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+        const uint32_t group = group0 + g;
+        const uint32_t t0 = (group << kappa) | ruler_slot(group, salt, kmask);
+        // the ruler switch belongs to its even-side walker; the claim returns both P values
+        const unsigned long long w0 = atomicAnd(S8 + t0, ((unsigned long long)((2u * group - rho_base) << 1) << cshift) | low_ones);
+        q[2 * g] = BENES_GUARD(__ldcg(Q + base + ((uint32_t(w0 >> m) & mmask) ^ 1u)), mmask);     // needs P[2 t0 + 1]
+        q[2 * g + 1] = BENES_GUARD(__ldcg(Q + base + ((uint32_t(w0) & mmask) ^ 1u)), mmask);      // needs P[2 t0]
+        fwd[2 * g] = 2u * t0; fwd[2 * g + 1] = 2u * t0 + 1u;
+        part[2 * g] = part[2 * g + 1] = kUnowned;
+        peer[2 * g] = (2u * group) ^ 1u; peer[2 * g + 1] = 2u * group;
+    }
+    uint32_t active = (1u << W) - 1u, hops = 0;
+    while (active) {
+        if (++hops > cap) {
+            *gate = 1u;
+            break;
+        }
+        if ((hops & 63u) == 0u && gate_raised(gate)) break;         // the level is relabelled anyway
+        unsigned long long w[W];
+#pragma unroll
+        for (int i = 0; i < W; ++i) {
+            w[i] = 0ull;
+            if (!((active >> i) & 1u)) continue;
+            const uint32_t j = base + q[i], t = j >> 1, side = j & 1u, g = t >> kappa;
+            if ((t & kmask) == ruler_slot(g, salt, kmask)) {        // reached the next ruler
+                peer[i] = (2u * g + side) ^ 1u;
+                active &= ~(1u << i);
+            } else {
+                w[i] = atomicAnd(S8 + t, ((unsigned long long)((((rho0 + i) - rho_base) << 1) | side) << cshift) | low_ones);
+            }
+        }
+        uint32_t qn[W];
+#pragma unroll
+        for (int i = 0; i < W; ++i) {
+            qn[i] = 0u;
+            if (!((active >> i) & 1u)) continue;
+            const uint32_t side = q[i] & 1u;                        // base is even
+            const uint32_t p = uint32_t(w[i] >> (side ? 0 : m)) & mmask;
+            qn[i] = BENES_GUARD(__ldcg(Q + base + (p ^ 1u)), mmask);
+        }
+#pragma unroll
+        for (int i = 0; i < W; ++i) {
+            if (!((active >> i) & 1u)) continue;
+            const uint32_t j = base + q[i];
+            const uint32_t prev = uint32_t(w[i] >> cshift);
+            if (prev != none8) {                                    // met the walker from the other end
+                __stcg(S8 + (j >> 1), w[i]);                        // put its code back
+                peer[i] = rho_base + (prev >> 1);
+                active &= ~(1u << i);
+            } else {
+                fwd[i] = min(fwd[i], j);
+                part[i] = min(part[i], j ^ 1u);
+                q[i] = qn[i];
+            }
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < W; ++i) rec[rho0 + i] = make_uint4(fwd[i], part[i], peer[i], 0u);
+}
+
 // Step 3.
 __global__ void __launch_bounds__(kThreads)
 k_combine(const uint4 *__restrict__ rec, unsigned long long *__restrict__ W, uint32_t rulers) {
@@ -571,13 +655,21 @@ int sampled_scratch_reset(const SampledScratch &sc, size_t total, int kappa, cud
 
 int sampled_label(void *S, bool packed, const uint32_t *Q, void *Sn, bool next_packed,
                   const SampledScratch &sc, size_t total, int log2m, int kappa, uint32_t salt,
-                  uint32_t cap, BitsLayout L, int out_stage, uint32_t *gate, cudaStream_t s) {
+                  uint32_t cap, int walk_pairs, BitsLayout L, int out_stage, uint32_t *gate, cudaStream_t s) {
     const uint32_t R = uint32_t(total >> kappa);
     const unsigned rgrid = (R + kThreads - 1) / kThreads;
     {
         ProfileScope ps(kWalk, s);
         const unsigned wgrid = (R + kWalkThreads - 1) / kWalkThreads;
-        if (packed) k_walk<true><<<wgrid, kWalkThreads, 0, s>>>(S, Q, sc.rec, R, log2m, kappa, salt, cap, gate);
+        // Two walkers per thread pay once the halved number of threads still fills the GPU
+        // (C4, cache-resident levels: 0.52-0.57 instead of 0.55-0.63 ms); below that the launch
+        // lasts as long as its longest thread and one walker per thread is faster.  Four and
+        // eight walkers per thread measured slower (0.60 and 0.90 ms).
+        const bool pair = walk_pairs == 2 || (walk_pairs == 1 && size_t(R >> 1) >= size_t(sm_count()) * 2048);
+        if (packed && pair)
+            k_walk_multi<1><<<((R >> 1) + kWalkThreads - 1) / kWalkThreads, kWalkThreads, 0, s>>>(
+                static_cast<unsigned long long *>(S), Q, sc.rec, R >> 1, log2m, kappa, salt, cap, gate);
+        else if (packed) k_walk<true><<<wgrid, kWalkThreads, 0, s>>>(S, Q, sc.rec, R, log2m, kappa, salt, cap, gate);
         else k_walk<false><<<wgrid, kWalkThreads, 0, s>>>(S, Q, sc.rec, R, log2m, kappa, salt, cap, gate);
         int rc = launch_status();
         if (rc) return rc;

@@ -27,7 +27,8 @@ def checked_library():
 
 @pytest.fixture
 def options():
-    keys = (binding.OPT_SAMPLE_LOG2K, binding.OPT_WALK_CAP, binding.OPT_CLUSTER, binding.OPT_INVERSE_PARTITIONED)
+    keys = (binding.OPT_SAMPLE_LOG2K, binding.OPT_WALK_CAP, binding.OPT_CLUSTER, binding.OPT_INVERSE_PARTITIONED,
+            binding.OPT_WALK_PAIRS)
     old = [binding.benes_get_option(k) for k in keys]
     yield
     for k, v in zip(keys, old):
@@ -99,6 +100,12 @@ def test_no_guard_fires_with_resampled_lists_bucketed_inverse_and_clusters(optio
         perm = inputs.random_perm_batch(n, batch, seed0=44)
         assert np.array_equal(route(perm, n), oracle.route(perm, n))
         assert_clean("clusters n=%d" % n)
+    binding.benes_set_option(binding.OPT_CLUSTER, 0)
+    binding.benes_set_option(binding.OPT_WALK_PAIRS, 2)
+    for n, batch in ((17, 3), (19, 1)):
+        perm = inputs.random_perm_batch(n, batch, seed0=45)
+        assert np.array_equal(route(perm, n), oracle.route(perm, n))
+        assert_clean("two walks per thread n=%d" % n)
 
 
 @pytest.mark.parametrize("n", [6, 14, 17, 22])

@@ -108,6 +108,27 @@ def test_route_every_ruler_spacing(kappa, labelling_options):
     assert np.array_equal(gpu_route(perm, 16), oracle.route(perm, 16))
 
 
+@pytest.mark.parametrize("mode", [0, 2])
+@pytest.mark.parametrize("kappa,cap", [(None, None), (2, None), (5, None), (None, 3)])
+def test_route_one_or_two_walks_per_thread(mode, kappa, cap, labelling_options):
+    """At packed levels a thread advances one walk or the two walks of a ruler switch
+    (the default picks by size; both forced here at sizes that take either)."""
+    w0 = binding.benes_get_option(binding.OPT_WALK_PAIRS)
+    binding.benes_set_option(binding.OPT_WALK_PAIRS, mode)
+    try:
+        if kappa is not None:
+            binding.benes_set_option(binding.OPT_SAMPLE_LOG2K, kappa)
+        if cap is not None:
+            binding.benes_set_option(binding.OPT_WALK_CAP, cap)
+        for n, batch in ((16, 3), (18, 1), (20, 1), (19, 5)):
+            perm = inputs.random_perm_batch(n, batch, seed0=300 + n) if batch > 1 else inputs.random_perm(n, 300 + n)
+            assert np.array_equal(gpu_route(perm, n), oracle.route(perm, n)), (n, batch)
+        for kind, perm in inputs.structured_perms(17).items():
+            assert np.array_equal(gpu_route(perm, 17), oracle.route(perm, 17)), kind
+    finally:
+        binding.benes_set_option(binding.OPT_WALK_PAIRS, w0)
+
+
 @pytest.fixture
 def cluster_mode():
     c0 = binding.benes_get_option(binding.OPT_CLUSTER)
