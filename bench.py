@@ -546,6 +546,8 @@ def run_gpu(args):
         binding.benes_set_option(binding.OPT_CLUSTER, args.cluster)
     if args.apply_fused is not None:
         binding.benes_set_option(binding.OPT_APPLY_FUSED, args.apply_fused)
+    if args.walk_pairs is not None:
+        binding.benes_set_option(binding.OPT_WALK_PAIRS, args.walk_pairs)
 
     name = args.workload
     stream = torch.cuda.Stream()
@@ -734,6 +736,8 @@ def main():
                     help="1: blocks of 2^16 finished by clusters of two CTAs; 0: blocks of 2^15 in one CTA")
     ap.add_argument("--apply-fused", type=int, default=None,
                     help="0: one payload-apply kernel per stage; 1: several stages per pass (default)")
+    ap.add_argument("--walk-pairs", type=int, default=None,
+                    help="ruler walks per thread: 0 one, 1 two where it pays (default), 2 two wherever possible")
     ap.add_argument("--rank-check", action="store_true",
                     help="run only the rank plumbing on the CPU (gloo); used by the tests")
     args = ap.parse_args()
