@@ -616,8 +616,8 @@ def run_gpu(args):
         out_p = torch.empty_like(x_p).pin_memory()
 
         def e2e_step():
-            binding.benes_route_host(perm_p, n, batch, bits_p, stream)
-            binding.benes_apply_host(bits_p, x_p, out_p, ebytes, n, batch, stream)
+            # one call: permutation and payload in, switch words and routed payload out
+            binding.benes_route_apply_host(perm_p, x_p, out_p, ebytes, n, batch, bits_p, stream)
 
         e2e_step()
         fence()
@@ -691,7 +691,8 @@ def run_gpu(args):
                        "ruler_spacing_log2": kappa},
             "clocks": clocks,
             "e2e": {"value": world * elems / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
-                    "h2d_bytes_per_step": case.perm_h.nbytes + bits_bytes + case.x_h.nbytes,
+                    "api": "benes_route_apply_host (pinned host buffers; switch words returned too)",
+                    "h2d_bytes_per_step": case.perm_h.nbytes + case.x_h.nbytes,
                     "d2h_bytes_per_step": bits_bytes + case.x_h.nbytes},
             "gpu_launches": launches,
             "roofline": roofline,

@@ -165,6 +165,18 @@ int benes_route_host(const uint32_t *perm_host, int log2n, int batch, uint32_t *
 int benes_apply_host(const uint32_t *switch_bits_host, const void *in_host, void *out_host,
                      int elem_bytes, int log2n, int batch, benes_stream_t stream);
 
+/*
+ * Both steps for host buffers in one call: out_host[b][j] = in_host[b][pi_b[j]].
+ * switch_bits_host may be NULL if the settings themselves are not wanted.  For
+ * batch * N >= 2^23 the payload travels to the device while the levels run, the
+ * finished stages and the finished parts of the routed payload travel back on a
+ * second copy stream, and the switch words never make the round trip through
+ * host memory that calling benes_route_host and benes_apply_host one after the
+ * other costs.  Synchronises `stream` before returning.
+ */
+int benes_route_apply_host(const uint32_t *perm_host, const void *in_host, void *out_host, int elem_bytes,
+                           int log2n, int batch, uint32_t *switch_bits_host, benes_stream_t stream);
+
 /* Number of 32-bit words of switch_bits for (log2n, batch); 0 on bad arguments. */
 size_t benes_switch_words(int log2n, int batch);
 

@@ -37,6 +37,7 @@ SYMBOLS = {
     "benes_apply_padded": (_i, [_vp, _vp, _vp, _i, _sz, _i, _vp]),
     "benes_route_host": (_i, [_vp, _i, _i, _vp, _vp]),
     "benes_apply_host": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp]),
+    "benes_route_apply_host": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _vp]),
     "benes_switch_words": (_sz, [_i, _i]),
     "benes_route_workspace_bytes": (_sz, [_i, _i]),
     "benes_apply_workspace_bytes": (_sz, [_i, _i, _i]),
@@ -199,6 +200,14 @@ def benes_apply_host(switch_bits_host, in_host, out_host, elem_bytes: int, log2n
     _check(load().benes_apply_host(_host_ptr(switch_bits_host, "switch_bits_host"),
                                    _host_ptr(in_host, "in_host"), _host_ptr(out_host, "out_host"),
                                    elem_bytes, log2n, batch, _stream(stream)), "benes_apply_host")
+
+
+def benes_route_apply_host(perm_host, in_host, out_host, elem_bytes: int, log2n: int, batch: int,
+                           switch_bits_host=None, stream=None) -> None:
+    bits = None if switch_bits_host is None else _host_ptr(switch_bits_host, "switch_bits_host")
+    _check(load().benes_route_apply_host(_host_ptr(perm_host, "perm_host"), _host_ptr(in_host, "in_host"),
+                                         _host_ptr(out_host, "out_host"), elem_bytes, log2n, batch, bits,
+                                         _stream(stream)), "benes_route_apply_host")
 
 
 def benes_set_workspace(buf, nbytes: int = 0) -> None:

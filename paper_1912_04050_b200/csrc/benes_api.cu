@@ -125,7 +125,10 @@ constexpr int kMaxPieces = 8;
 static_assert(kMaxPieces >= kApplyMaxParts, "the host pipe's events serve the apply parts too");
 struct HostPipe {
     uint32_t *bits_host = nullptr;     // finished stages go here (same layout as `bits`)
-    cudaStream_t side = nullptr;
+    cudaStream_t side = nullptr;       // host -> device copies
+    cudaStream_t back = nullptr;       // a second stream for device -> host copies (benes_route_apply_host)
+    cudaStream_t d2h = nullptr;        // where this call's finished stages leave: `side` or `back`
+    cudaEvent_t part_ready[kApplyMaxParts] = {};   // parts of a payload that have arrived
     int pieces = 0;                    // the permutation arrives in this many equal pieces
     cudaEvent_t piece_ready[kMaxPieces] = {};
     cudaEvent_t stage_ready[kMaxLevels] = {};
@@ -230,9 +233,9 @@ int route_levels(const uint32_t *perm, int n, size_t batch, uint32_t *bits, char
         if (hp && hp->bits_host) {
             // stages `level` and `out_stage` are final: send them home behind the computation
             BENES_CUDA_TRY(cudaEventRecord(hp->stage_ready[level], s));
-            BENES_CUDA_TRY(cudaStreamWaitEvent(hp->side, hp->stage_ready[level], 0));
-            if ((rc = copy_stage_rows(*hp, bits, n, batch, level, 1, hp->side))) return rc;
-            if ((rc = copy_stage_rows(*hp, bits, n, batch, out_stage, 1, hp->side))) return rc;
+            BENES_CUDA_TRY(cudaStreamWaitEvent(hp->d2h, hp->stage_ready[level], 0));
+            if ((rc = copy_stage_rows(*hp, bits, n, batch, level, 1, hp->d2h))) return rc;
+            if ((rc = copy_stage_rows(*hp, bits, n, batch, out_stage, 1, hp->d2h))) return rc;
         }
     }
     const int records = rec_is_packed(fused_m, kappa) ? 2 : 1;
@@ -257,10 +260,12 @@ int route_levels(const uint32_t *perm, int n, size_t batch, uint32_t *bits, char
         const size_t w = stage_words(n) * 4, col1 = (b1 << (fused_m - 6)) * 4;
         char *dst = reinterpret_cast<char *>(hp->bits_host) + size_t(first) * w;
         const char *src = reinterpret_cast<const char *>(bits) + size_t(first) * w;
-        BENES_CUDA_TRY(cudaStreamWaitEvent(hp->side, hp->stage_ready[kMaxLevels - 2], 0));
-        BENES_CUDA_TRY(cudaMemcpy2DAsync(dst, w, src, w, col1, size_t(rows), cudaMemcpyDeviceToHost, hp->side));
+        BENES_CUDA_TRY(cudaStreamWaitEvent(hp->d2h, hp->stage_ready[kMaxLevels - 2], 0));
+        BENES_CUDA_TRY(cudaMemcpy2DAsync(dst, w, src, w, col1, size_t(rows), cudaMemcpyDeviceToHost, hp->d2h));
+        BENES_CUDA_TRY(cudaEventRecord(hp->stage_ready[kMaxLevels - 3], s));
+        BENES_CUDA_TRY(cudaStreamWaitEvent(hp->d2h, hp->stage_ready[kMaxLevels - 3], 0));
         BENES_CUDA_TRY(cudaMemcpy2DAsync(dst + col1, w, src + col1, w, w - col1, size_t(rows),
-                                         cudaMemcpyDeviceToHost, s));
+                                         cudaMemcpyDeviceToHost, hp->d2h));
         return BENES_OK;
     }
     {
@@ -284,6 +289,8 @@ int host_pipe_for_current_device(HostPipe **out) {
     HostPipe &hp = pipes[dev];
     if (!ready[dev]) {
         BENES_CUDA_TRY(cudaStreamCreateWithFlags(&hp.side, cudaStreamNonBlocking));
+        BENES_CUDA_TRY(cudaStreamCreateWithFlags(&hp.back, cudaStreamNonBlocking));
+        for (cudaEvent_t &e : hp.part_ready) BENES_CUDA_TRY(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
         for (cudaEvent_t &e : hp.piece_ready) BENES_CUDA_TRY(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
         for (cudaEvent_t &e : hp.stage_ready) BENES_CUDA_TRY(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
         ready[dev] = true;
@@ -481,6 +488,7 @@ int benes_route_host(const uint32_t *perm_host, int log2n, int batch, uint32_t *
         if ((rc = host_pipe_for_current_device(&hp))) return rc;
         const size_t T = size_t(batch) << n;
         hp->bits_host = switch_bits_host;
+        hp->d2h = hp->side;
         hp->pieces = (T >= (size_t(1) << 23)) ? kMaxPieces : 1;
         // the side stream must not touch the workspace before earlier work on `s` is done
         BENES_CUDA_TRY(cudaEventRecord(hp->stage_ready[kMaxLevels - 1], s));
@@ -557,6 +565,84 @@ int benes_apply_host(const uint32_t *switch_bits_host, const void *in_host, void
     BENES_CUDA_TRY(cudaMemcpyAsync(out_host, d_out, data_bytes, cudaMemcpyDeviceToHost, s));
     BENES_CUDA_TRY(cudaStreamSynchronize(s));
     return BENES_OK;
+}
+
+int benes_route_apply_host(const uint32_t *perm_host, const void *in_host, void *out_host, int elem_bytes,
+                           int log2n, int batch, uint32_t *switch_bits_host, benes_stream_t stream) {
+    if (!perm_host || !in_host || !out_host || bad_shape(log2n, batch)) return BENES_ERR_BADARG;
+    if (elem_bytes != 4 && elem_bytes != 8) return BENES_ERR_BADARG;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    const int n = log2n;
+    const Options opt = options();
+    const size_t T = size_t(batch) << n;
+    const size_t data_bytes = T * size_t(elem_bytes);
+    const size_t chunks = apply_fused_chunks(n, size_t(batch));
+    const bool piped = n > kFusedLog2M && level_chunk(n, size_t(batch), opt.chunk_log2) == size_t(batch) &&
+                       opt.apply_fused && T >= (size_t(1) << 23) && chunks > 0 && chunks % kApplyMaxParts == 0;
+    if (!piped) {
+        // small or chunked inputs: one call after the other (the switch words stay on the host side
+        // of the first call only if the caller wants them)
+        const size_t words = benes_switch_words(n, batch);
+        uint32_t *bits_tmp = switch_bits_host;
+        if (!bits_tmp) {
+            if (cudaMallocHost(&bits_tmp, words * 4) != cudaSuccess) { cudaGetLastError(); return BENES_ERR_NOMEM; }
+        }
+        int rc = benes_route_host(perm_host, n, batch, bits_tmp, stream);
+        if (!rc) rc = benes_apply_host(bits_tmp, in_host, out_host, elem_bytes, n, batch, stream);
+        if (!switch_bits_host) cudaFreeHost(bits_tmp);
+        return rc;
+    }
+    const size_t perm_bytes = T * 4, bits_bytes = benes_switch_words(n, batch) * 4;
+    const size_t route_ws = align_up(route_ws_bytes(n, size_t(batch)));
+    const size_t apply_ws = align_up(apply_ws_bytes(elem_bytes, n, size_t(batch)));
+    void *ws = nullptr;
+    int rc = get_workspace(route_ws + apply_ws + align_up(perm_bytes) + align_up(bits_bytes) + 2 * align_up(data_bytes), &ws);
+    if (rc) return rc;
+    char *base = static_cast<char *>(ws);
+    char *scratch = base + route_ws;
+    uint32_t *d_perm = reinterpret_cast<uint32_t *>(scratch + apply_ws);
+    uint32_t *d_bits = reinterpret_cast<uint32_t *>(reinterpret_cast<char *>(d_perm) + align_up(perm_bytes));
+    char *d_in = reinterpret_cast<char *>(d_bits) + align_up(bits_bytes);
+    char *d_out = d_in + align_up(data_bytes);
+    HostPipe *hp = nullptr;
+    if ((rc = host_pipe_for_current_device(&hp))) return rc;
+    hp->bits_host = switch_bits_host;              // null: the switch words stay on the device
+    hp->d2h = hp->back;
+    hp->pieces = kMaxPieces;
+    // the copy streams must not touch the workspace before earlier work on `s` is done
+    BENES_CUDA_TRY(cudaEventRecord(hp->stage_ready[kMaxLevels - 1], s));
+    BENES_CUDA_TRY(cudaStreamWaitEvent(hp->side, hp->stage_ready[kMaxLevels - 1], 0));
+    BENES_CUDA_TRY(cudaStreamWaitEvent(hp->back, hp->stage_ready[kMaxLevels - 1], 0));
+    // inbound: the permutation in pieces, then the payload in parts, behind one another on one
+    // stream, while the levels run; outbound (second stream): finished stages, then finished parts
+    const size_t per = perm_bytes / size_t(hp->pieces);
+    for (int i = 0; i < hp->pieces; ++i) {
+        BENES_CUDA_TRY(cudaMemcpyAsync(reinterpret_cast<char *>(d_perm) + per * size_t(i),
+                                       reinterpret_cast<const char *>(perm_host) + per * size_t(i), per,
+                                       cudaMemcpyHostToDevice, hp->side));
+        BENES_CUDA_TRY(cudaEventRecord(hp->piece_ready[i], hp->side));
+    }
+    ApplyHostPipe pipe;
+    pipe.parts = kApplyMaxParts;
+    pipe.side = hp->back;
+    pipe.out_host = out_host;
+    const size_t part = data_bytes / size_t(pipe.parts);
+    for (int i = 0; i < pipe.parts; ++i) {
+        BENES_CUDA_TRY(cudaMemcpyAsync(d_in + part * size_t(i), static_cast<const char *>(in_host) + part * size_t(i),
+                                       part, cudaMemcpyHostToDevice, hp->side));
+        BENES_CUDA_TRY(cudaEventRecord(hp->part_ready[i], hp->side));
+        pipe.in_ready[i] = hp->part_ready[i];
+    }
+    rc = route_levels(d_perm, n, size_t(batch), d_bits, base, s, opt, hp);
+    if (!rc) {
+        // the route no longer waits on these events; the apply's last pass reuses them
+        for (int i = 0; i < pipe.parts; ++i) pipe.out_done[i] = hp->stage_ready[i];
+        ProfileScope ps(kApplyFused, s);
+        rc = launch_apply_fused(d_bits, d_in, d_out, scratch, elem_bytes, n, size_t(batch), s, &pipe);
+    }
+    cudaError_t e1 = cudaStreamSynchronize(s), e2 = cudaStreamSynchronize(hp->side), e3 = cudaStreamSynchronize(hp->back);
+    if (rc) return rc;
+    return (e1 == cudaSuccess && e2 == cudaSuccess && e3 == cudaSuccess) ? BENES_OK : BENES_ERR_CUDA;
 }
 
 int benes_validate_perm(const uint32_t *perm, int log2n, int batch, benes_stream_t stream) {

@@ -428,6 +428,31 @@ def test_host_entry_points(n, batch, pinned):
     assert np.array_equal(bits2, bits)
 
 
+@pytest.mark.parametrize("n,batch,dtype,want_bits", [(23, 1, np.uint64, True), (24, 1, np.uint32, True),
+                                                     (23, 2, np.uint64, False), (18, 3, np.uint64, True),
+                                                     (15, 2, np.uint32, False), (25, 1, np.uint64, True)])
+def test_route_apply_host_in_one_call(n, batch, dtype, want_bits):
+    """Permutation and payload in, routed payload (and, if wanted, the switch words) out; from
+    2^23 elements on the payload arrives while the levels run and the words never pass through
+    host memory."""
+    perm = inputs.random_perm_batch(n, batch, seed0=600 + n)
+    x = inputs.payload_u64(batch << n, 8).reshape(batch, -1)
+    if dtype == np.uint32:
+        x = (x >> np.uint64(32)).astype(np.uint32)
+    perm_t = torch.from_numpy(perm.view(np.int32)).pin_memory()
+    x_t = torch.from_numpy(x.view({4: np.int32, 8: np.int64}[x.dtype.itemsize])).pin_memory()
+    out_t = torch.full_like(x_t, -1).pin_memory()
+    bits_t = torch.full((batch, 2 * n - 1, (1 << n) // 64), 0x33333333, dtype=torch.int32).pin_memory() if want_bits else None
+    for _ in range(2):          # the second call reuses streams, events and the workspace
+        out_t.fill_(-1)
+        binding.benes_route_apply_host(perm_t, x_t, out_t, x.dtype.itemsize, n, batch, bits_t)
+        assert np.array_equal(out_t.numpy().view(dtype), np.take_along_axis(x, perm.astype(np.int64), axis=1))
+    if want_bits:
+        want = oracle.route(perm, n) if n <= 24 else gpu_route(perm, n)
+        assert np.array_equal(bits_t.numpy().view(np.uint32), want)
+    binding.benes_release_workspace()
+
+
 def test_route_host_split_tail_matches_device_path():
     """From 592 blocks of 2^15 on (N = 2^25 here) the host entry point finishes the
     in-CTA levels in two launches and copies the first one's columns home while the
