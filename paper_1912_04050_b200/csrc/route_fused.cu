@@ -52,6 +52,71 @@ __device__ __forceinline__ uint32_t fused_slot(uint32_t group, uint32_t salt) {
     return ((group + salt * 0x632BE5ABu) * 0x9E3779B1u) >> (32 - kFKappa);
 }
 
+// The last five levels of one group of 32 outputs (sub-blocks of 32 and less stay
+// inside it): a warp finishes the group in registers, one output per lane, p = the
+// lane's entry of the group's sub-permutation, gathers done with shuffles (the
+// inverse goes through the group's 32 entries of Q, which only this warp touches).
+// grp = index of the group in the CTA's block, g0 = 32 grp.
+template <int LOGM>
+__device__ __forceinline__ void fused_tail32(uint32_t p, int grp, int g0, int lane, uint16_t *Q, uint32_t *my_bits,
+                                             int n, int level0, size_t stage_w) {
+    constexpr int M = 1 << LOGM;
+    uint16_t *half = reinterpret_cast<uint16_t *>(my_bits);     // 16 switches = one half word
+    const size_t half_stride = stage_w * 2;
+#pragma unroll
+    for (int ls = 5; ls >= 2; --ls) {
+        const uint32_t sm_ = (1u << ls) - 1u, sbl = uint32_t(lane) & ~sm_;
+        const int lvl = level0 + (LOGM - ls);
+        p &= sm_;
+        // a1: inverse inside the sub-block
+        Q[g0 + sbl + p] = uint16_t(uint32_t(lane) & sm_);
+        __syncwarp();
+        const uint32_t q = Q[g0 + lane];
+        __syncwarp();
+        // a2: successor
+        const uint32_t p1 = __shfl_xor_sync(0xFFFFFFFFu, p, 1);
+        uint32_t nxt = sbl + __shfl_sync(0xFFFFFFFFu, q, int(sbl + (p1 ^ 1u)));
+        uint32_t mn = uint32_t(lane);
+        // a3: synchronous pointer jumping, ls-1 passes cover cycles of 2^(ls-1)
+#pragma unroll
+        for (int r = 0; r < ls - 1; ++r) {
+            const uint32_t mm = __shfl_sync(0xFFFFFFFFu, mn, int(nxt));
+            nxt = __shfl_sync(0xFFFFFFFFu, nxt, int(nxt));
+            mn = min(mn, mm);
+        }
+        const uint32_t c = mn & 1u;                          // a4, every output
+        // output side of a5: switch t = lane (< 16) takes the colour of output 2t
+        const uint32_t ce = __shfl_sync(0xFFFFFFFFu, c, (lane & 15) * 2);
+        const uint32_t outw = __ballot_sync(0xFFFFFFFFu, ce) & 0xFFFFu;
+        // input side of a5: colour of the output fed by input 2t
+        const uint32_t qe = __shfl_sync(0xFFFFFFFFu, q, (lane & 15) * 2);
+        const uint32_t sbe = uint32_t((lane & 15) * 2) & ~sm_;
+        const uint32_t ci = __shfl_sync(0xFFFFFFFFu, c, int(sbe + qe));
+        const uint32_t inw = __ballot_sync(0xFFFFFFFFu, ci) & 0xFFFFu;
+        if (lane == 0) {
+            if (M == 32) {
+                my_bits[size_t(2 * n - 2 - lvl) * stage_w] = outw;
+                my_bits[size_t(lvl) * stage_w] = inw;
+            } else {
+                half[size_t(2 * n - 2 - lvl) * half_stride + grp] = uint16_t(outw);
+                half[size_t(lvl) * half_stride + grp] = uint16_t(inw);
+            }
+        }
+        // a6: position dl of the upper (lower) half takes the colour-0 (1) output of switch tl
+        const uint32_t H = 1u << (ls - 1), dl = uint32_t(lane) & sm_;
+        const uint32_t tl = dl & (H - 1u), lower = dl >> (ls - 1);
+        const uint32_t c2 = __shfl_sync(0xFFFFFFFFu, c, int(sbl + 2u * tl));
+        p = __shfl_sync(0xFFFFFFFFu, p, int(sbl + 2u * tl + (c2 ^ lower))) >> 1;
+    }
+    // a7: middle stage
+    const uint32_t pm = __shfl_sync(0xFFFFFFFFu, p, (lane & 15) * 2) & 1u;
+    const uint32_t midw = __ballot_sync(0xFFFFFFFFu, pm) & 0xFFFFu;
+    if (lane == 0) {
+        if (M == 32) my_bits[size_t(n - 1) * stage_w] = midw;
+        else half[size_t(n - 1) * half_stride + grp] = uint16_t(midw);
+    }
+}
+
 // Levels level0 .. level0 + LOGM - 1 of the block of M = 2^LOGM outputs whose
 // sub-permutation (16-bit, local) is in Pcur.  Pnext is the other buffer of M
 // entries; `tail` = the extra scratch bytes (FusedCfg::kExtra); my_bits = where the
@@ -76,69 +141,57 @@ __device__ __forceinline__ void fused_levels(uint16_t *Pcur, uint16_t *Pnext, ui
         const uint32_t smask = S - 1u;
         const int level = level0 + k;
 
-        if (logS == 5 && LOGM >= 5) {
-            // Sub-blocks of 32 and less stay inside one group of 32 outputs for all
-            // remaining levels: a warp finishes a group in registers, one output
-            // per lane, gathers done with shuffles (the inverse goes through 32
-            // entries of Q, which only this warp touches).
-            uint16_t *half = reinterpret_cast<uint16_t *>(my_bits);     // 16 switches = one half word
-            const size_t half_stride = stage_w * 2;
-            for (int grp = tid >> 5; grp < M / 32; grp += T / 32) {
-                const int g0 = grp * 32;
-                uint32_t p = BENES_GUARD(uint32_t(Pcur[g0 + lane]), 31u);                      // local to the 32-sub-block
+        if (logS == 6 && LOGM >= 6) {
+            // Sub-blocks of 64: a warp takes one, a lane one of its 32 switches (two outputs),
+            // and labels it in registers: the (next, min) words of a lane's two outputs share
+            // one register (8 + 8 bits each), a jump is one shuffle per output, five passes
+            // cover cycles of 32 outputs.  The two half-blocks then stay in the warp for the
+            // remaining levels (fused_tail32), so nothing of these six levels but the inverse
+            // goes through shared memory and no CTA-wide barrier is needed any more.
+            for (int g64 = tid >> 5; g64 < M / 64; g64 += T / 32) {
+                const int g0 = g64 * 64;
+                const uint32_t pp = *reinterpret_cast<const uint32_t *>(Pcur + g0 + 2 * lane);
+                const uint32_t p0 = BENES_GUARD16(pp, 63u), p1 = BENES_GUARD(pp >> 16, 63u);
+                // a1: inverse inside the sub-block
+                Q[g0 + p0] = uint16_t(2 * lane);
+                Q[g0 + p1] = uint16_t(2 * lane + 1);
+                __syncwarp();
+                const uint32_t q0 = BENES_GUARD(uint32_t(Q[g0 + 2 * lane]), 63u);   // output fed by input 2 lane
+                // a2: successors of the lane's two outputs
+                const uint32_t nx0 = BENES_GUARD(uint32_t(Q[g0 + (p1 ^ 1u)]), 63u);
+                const uint32_t nx1 = BENES_GUARD(uint32_t(Q[g0 + (p0 ^ 1u)]), 63u);
+                __syncwarp();                                            // the tails below reuse these entries of Q
+                uint32_t w = (nx0 | (uint32_t(2 * lane) << 8)) | ((nx1 | (uint32_t(2 * lane + 1) << 8)) << 16);
+                // a3: synchronous pointer jumping
 #pragma unroll
-                for (int ls = 5; ls >= 2; --ls) {
-                    const uint32_t sm_ = (1u << ls) - 1u, sbl = uint32_t(lane) & ~sm_;
-                    const int lvl = level0 + (LOGM - ls);
-                    p &= sm_;
-                    // a1: inverse inside the sub-block
-                    Q[g0 + sbl + p] = uint16_t(uint32_t(lane) & sm_);
-                    __syncwarp();
-                    const uint32_t q = Q[g0 + lane];
-                    __syncwarp();
-                    // a2: successor
-                    const uint32_t p1 = __shfl_xor_sync(0xFFFFFFFFu, p, 1);
-                    uint32_t nxt = sbl + __shfl_sync(0xFFFFFFFFu, q, int(sbl + (p1 ^ 1u)));
-                    uint32_t mn = uint32_t(lane);
-                    // a3: synchronous pointer jumping, ls-1 passes cover cycles of 2^(ls-1)
-#pragma unroll
-                    for (int r = 0; r < ls - 1; ++r) {
-                        const uint32_t mm = __shfl_sync(0xFFFFFFFFu, mn, int(nxt));
-                        nxt = __shfl_sync(0xFFFFFFFFu, nxt, int(nxt));
-                        mn = min(mn, mm);
-                    }
-                    const uint32_t c = mn & 1u;                          // a4, every output
-                    // output side of a5: switch t = lane (< 16) takes the colour of output 2t
-                    const uint32_t ce = __shfl_sync(0xFFFFFFFFu, c, (lane & 15) * 2);
-                    const uint32_t outw = __ballot_sync(0xFFFFFFFFu, ce) & 0xFFFFu;
-                    // input side of a5: colour of the output fed by input 2t
-                    const uint32_t qe = __shfl_sync(0xFFFFFFFFu, q, (lane & 15) * 2);
-                    const uint32_t sbe = uint32_t((lane & 15) * 2) & ~sm_;
-                    const uint32_t ci = __shfl_sync(0xFFFFFFFFu, c, int(sbe + qe));
-                    const uint32_t inw = __ballot_sync(0xFFFFFFFFu, ci) & 0xFFFFu;
-                    if (lane == 0) {
-                        if (M == 32) {
-                            my_bits[size_t(2 * n - 2 - lvl) * stage_w] = outw;
-                            my_bits[size_t(lvl) * stage_w] = inw;
-                        } else {
-                            half[size_t(2 * n - 2 - lvl) * half_stride + grp] = uint16_t(outw);
-                            half[size_t(lvl) * half_stride + grp] = uint16_t(inw);
-                        }
-                    }
-                    // a6: position dl of the upper (lower) half takes the colour-0 (1) output of switch tl
-                    const uint32_t H = 1u << (ls - 1), dl = uint32_t(lane) & sm_;
-                    const uint32_t tl = dl & (H - 1u), lower = dl >> (ls - 1);
-                    const uint32_t c2 = __shfl_sync(0xFFFFFFFFu, c, int(sbl + 2u * tl));
-                    p = __shfl_sync(0xFFFFFFFFu, p, int(sbl + 2u * tl + (c2 ^ lower))) >> 1;
+                for (int r = 0; r < 5; ++r) {
+                    const uint32_t a0 = w & 0xFFu, a1 = (w >> 16) & 0xFFu;
+                    const uint32_t v0 = (__shfl_sync(0xFFFFFFFFu, w, int(a0 >> 1)) >> ((a0 & 1u) * 16u)) & 0xFFFFu;
+                    const uint32_t v1 = (__shfl_sync(0xFFFFFFFFu, w, int(a1 >> 1)) >> ((a1 & 1u) * 16u)) & 0xFFFFu;
+                    const uint32_t n0 = (v0 & 0xFFu) | min(w & 0xFF00u, v0 & 0xFF00u);
+                    const uint32_t n1 = (v1 & 0xFFu) | min((w >> 16) & 0xFF00u, v1 & 0xFF00u);
+                    w = n0 | (n1 << 16);
                 }
-                // a7: middle stage
-                const uint32_t pm = __shfl_sync(0xFFFFFFFFu, p, (lane & 15) * 2) & 1u;
-                const uint32_t midw = __ballot_sync(0xFFFFFFFFu, pm) & 0xFFFFu;
+                const uint32_t c0 = (w >> 8) & 1u;                       // a4: colour of output 2 lane (2 lane + 1 has the other)
+                // a5: output side, switch = lane; input side, the colour of the output fed by input 2 lane
+                const uint32_t outw = __ballot_sync(0xFFFFFFFFu, c0);
+                const uint32_t ci = (__shfl_sync(0xFFFFFFFFu, c0, int(q0 >> 1)) ^ q0) & 1u;
+                const uint32_t inw = __ballot_sync(0xFFFFFFFFu, ci);
                 if (lane == 0) {
-                    if (M == 32) my_bits[size_t(n - 1) * stage_w] = midw;
-                    else half[size_t(n - 1) * half_stride + grp] = uint16_t(midw);
+                    my_bits[size_t(2 * n - 2 - level) * stage_w + g64] = outw;
+                    my_bits[size_t(level) * stage_w + g64] = inw;
                 }
+                // a6: position `lane` of the upper (lower) half takes the colour-0 (1) output of switch `lane`
+                fused_tail32<LOGM>((c0 ? p1 : p0) >> 1, 2 * g64, g0, lane, Q, my_bits, n, level0, stage_w);
+                fused_tail32<LOGM>((c0 ? p0 : p1) >> 1, 2 * g64 + 1, g0 + 32, lane, Q, my_bits, n, level0, stage_w);
             }
+            break;
+        }
+
+        if (logS == 5 && LOGM >= 5) {
+            for (int grp = tid >> 5; grp < M / 32; grp += T / 32)
+                fused_tail32<LOGM>(BENES_GUARD(uint32_t(Pcur[grp * 32 + lane]), 31u), grp, grp * 32, lane, Q, my_bits, n,
+                                   level0, stage_w);
             break;
         }
 
