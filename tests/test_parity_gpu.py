@@ -129,6 +129,36 @@ def test_route_one_or_two_walks_per_thread(mode, kappa, cap, labelling_options):
         binding.benes_set_option(binding.OPT_WALK_PAIRS, w0)
 
 
+def test_route_random_option_combinations(labelling_options):
+    """Seeded draws over sizes, batches, input kinds and every option that changes the path
+    (ruler spacing, hop limit, walks per thread, clusters, inverse form, chunking): the bits never
+    depend on the path."""
+    rng = np.random.default_rng(2024)
+    keys = (binding.OPT_WALK_PAIRS, binding.OPT_CLUSTER, binding.OPT_INVERSE_PARTITIONED, binding.OPT_CHUNK_LOG2)
+    old = [binding.benes_get_option(k) for k in keys]
+    try:
+        for trial in range(48):
+            n = int(rng.integers(15, 21))
+            batch = int(rng.choice([1, 1, 2, 3, 5])) if n <= 18 else 1
+            kind = str(rng.choice(["random", "random", "random", "sattolo", "shift1", "bitrev", "identity"]))
+            opts = {binding.OPT_SAMPLE_LOG2K: int(rng.choice([0, 2, 3, 4, 4, 5, 6, 8])),
+                    binding.OPT_WALK_CAP: int(rng.choice([1, 7, 100, 1 << 14, 1 << 14])),
+                    binding.OPT_WALK_PAIRS: int(rng.integers(0, 3)),
+                    binding.OPT_CLUSTER: int(rng.integers(0, 2)),
+                    binding.OPT_INVERSE_PARTITIONED: int(rng.integers(0, 2)),
+                    binding.OPT_CHUNK_LOG2: int(rng.choice([30, 30, 17, 18]))}
+            for k, v in opts.items():
+                binding.benes_set_option(k, v)
+            if kind == "random":
+                perm = inputs.random_perm_batch(n, batch, seed0=5000 + trial)
+            else:
+                perm = np.tile(inputs.structured_perms(n)[kind], (batch, 1))
+            assert np.array_equal(gpu_route(perm, n), oracle.route(perm, n)), (trial, n, batch, kind, opts)
+    finally:
+        for k, v in zip(keys, old):
+            binding.benes_set_option(k, v)
+
+
 @pytest.fixture
 def cluster_mode():
     c0 = binding.benes_get_option(binding.OPT_CLUSTER)
