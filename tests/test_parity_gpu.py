@@ -552,6 +552,37 @@ def test_non_permutation_input_is_memory_safe(n):
     assert np.array_equal(gpu_route(perm, n), oracle.route(perm, n))
 
 
+@pytest.mark.parametrize("n,batch", [(12, 4), (18, 1), (20, 1)])
+def test_route_and_apply_replayed_from_a_cuda_graph(n, batch):
+    """Both entry points only enqueue work on the caller's stream (once the workspace exists and
+    the kernels' attributes are set, i.e. after one ordinary call), so a caller can capture them
+    into a CUDA graph and replay it on new contents of the same buffers."""
+    perm_a = inputs.random_perm_batch(n, batch, seed0=900 + n)
+    perm_b = inputs.random_perm_batch(n, batch, seed0=950 + n)
+    x = inputs.payload_u64(batch << n, 3).reshape(batch, -1)
+    d_perm, d_x = dev(perm_a), dev(x)
+    bits = torch.empty(binding.benes_switch_words(n, batch), dtype=torch.int32, device="cuda")
+    out = torch.empty_like(d_x)
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        binding.benes_route(d_perm, n, batch, bits, side)                  # warm-up: workspace, attributes
+        binding.benes_apply_ex(bits, d_x, out, 8, n, batch, side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        binding.benes_route(d_perm, n, batch, bits, torch.cuda.current_stream())
+        binding.benes_apply_ex(bits, d_x, out, 8, n, batch, torch.cuda.current_stream())
+    for perm in (perm_b, perm_a, perm_b):
+        d_perm.copy_(dev(perm))
+        bits.fill_(-1)
+        out.fill_(-1)
+        graph.replay()
+        torch.cuda.synchronize()
+        shape = (batch, 2 * n - 1, max(1, (1 << n) // 64))
+        assert np.array_equal(host(bits, np.uint32).reshape(shape), oracle.route(perm, n))
+        assert np.array_equal(host(out, np.uint64).reshape(x.shape), np.take_along_axis(x, perm.astype(np.int64), axis=1))
+
+
 def test_launch_counter_counts():
     n = 17
     before = binding.benes_launch_count()
