@@ -201,9 +201,22 @@ k_inverse_scatter_smem(const uint2 *__restrict__ pairs, uint32_t *__restrict__ Q
         piece[two[i].x & kInBucket] = BENES_GUARD(two[i].y, mmask);
         piece[two[i].z & kInBucket] = BENES_GUARD(two[i].w, mmask);
     }
+    // The finished piece leaves as ONE bulk asynchronous copy (shared -> global, 128 KiB, both
+    // ends 16-byte aligned: the piece starts the dynamic shared memory, its place in Q is a
+    // multiple of 128 KiB) issued by one thread: the copy engine streams it out while the
+    // SM's load/store slots stay free for the next CTA's scatter.  The writes above went
+    // through the generic proxy, hence the proxy fence before the barrier; the issuing
+    // thread waits until the engine has read the piece, so the CTA's shared memory is not
+    // handed to another CTA early (a hardware completion, not a flag to spin on).
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     __syncthreads();
-    uint4 *dst = reinterpret_cast<uint4 *>(Q + b0);
-    for (uint32_t k = threadIdx.x; k < kEntries / 4; k += 1024) dst[k] = reinterpret_cast<const uint4 *>(piece)[k];
+    if (threadIdx.x == 0) {
+        const uint32_t src = uint32_t(__cvta_generic_to_shared(piece));
+        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                     :: "l"(Q + b0), "r"(src), "r"(uint32_t(kEntries * 4)) : "memory");
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+    }
 }
 
 // Pass 2, buckets of 2^kBucketL2Log2 entries.
