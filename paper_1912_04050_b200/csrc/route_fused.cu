@@ -13,9 +13,12 @@
 //     list (M/8 words of (next, min), 16 + 16 bit) is labelled by in-place
 //     pointer jumping; a switch takes (minimum of its owner & 1) ^ side;
 //   - switches nobody claimed (loops without ruler) walk their own cycle;
-//   - sub-blocks of S <= 256 are labelled by in-place pointer jumping over all
-//     outputs with 16-bit words (next, min: 8 + 8 bit, local to the sub-block),
-//     which costs fewer instructions than walks once cycles are this short.
+//   - sub-blocks of S = 256 and 128 are labelled by in-place pointer jumping over
+//     all outputs with 16-bit words (next, min: 8 + 8 bit, local to the sub-block),
+//     which costs fewer instructions than walks once cycles are this short;
+//   - sub-blocks of S <= 64 never leave a warp: it labels a sub-block of 64 in
+//     registers (a switch per lane, jumps by shuffle) and both halves of it, down
+//     to the middle stage, one output per lane.
 // The scratch of the labelling (owners, walk records, list) lives where the
 // next level's P' is written afterwards.
 #include "common.cuh"

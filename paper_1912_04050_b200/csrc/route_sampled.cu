@@ -16,7 +16,9 @@
 //      owns: together they touch every switch of the segment once.  A walker
 //      keeps the smallest output index on its own side of the switches it
 //      claimed (fwd), the smallest on the far side (part), and its partner
-//      (peer).  The claim stores (walker, side of arrival).
+//      (peer).  The claim stores (walker, side of arrival).  At the levels with
+//      packed records and enough rulers to fill the GPU a thread advances the
+//      two walkers of one ruler switch together (k_walk_multi).
 //   3. k_combine: the segment of walker rho ends at ruler output peer^1 and
 //      its minimum is min(fwd[rho], part[peer]): one 64-bit (next, min) word
 //      per ruler output -- the contracted list.
