@@ -250,9 +250,14 @@ __device__ __forceinline__ void fused_levels(uint16_t *Pcur, uint16_t *Pnext, ui
                     pp = *reinterpret_cast<const uint32_t *>(Pcur + 2u * t);
                     p = BENES_GUARD16(side ? pp : (pp >> 16), smask);
                     const uint32_t qn = BENES_GUARD(uint32_t(Q[sb + (p ^ 1u)]), smask);
-                    const uint32_t prev = atomicCAS(reinterpret_cast<unsigned short *>(own + t),
-                                                    static_cast<unsigned short>(kNone16),
-                                                    static_cast<unsigned short>((uint32_t(rho) << 1) | side));
+                    // The claim needs no atomic.  Only the two walkers of this segment ever reach
+                    // switch t, from opposite ends.  If both find it free at the same moment, both
+                    // write (either code is a valid owner: the two stand for mirror cycles and
+                    // arrive on opposite sides, so the colour comes out the same), both go on, and
+                    // each stops at the next switch, which the other has claimed; minima are taken
+                    // over one switch more, which changes nothing.
+                    const uint32_t prev = reinterpret_cast<volatile uint16_t *>(own)[t];
+                    if (prev == kNone16) reinterpret_cast<volatile uint16_t *>(own)[t] = uint16_t((uint32_t(rho) << 1) | side);
                     if (prev != kNone16) {                                  // met the other walker
                         pr = prev >> 1;
                         break;
