@@ -26,8 +26,11 @@
  *
  * Conventions.  Every pointer is a DEVICE pointer unless the name says
  * "_host".  The caller owns every buffer it passes; the library owns only its
- * internal workspace (one per device, grown on demand with cudaMalloc on the
- * first call that needs it, or supplied by the caller).  Work is enqueued on
+ * internal workspace (one per device, or supplied by the caller).  A call that
+ * needs more than the workspace holds replaces it in stream order on `stream`
+ * (cudaFreeAsync + cudaMallocAsync from the device's default pool: no
+ * device-wide synchronisation; only on a device without memory pools the old
+ * cudaDeviceSynchronize + cudaFree + cudaMalloc).  Work is enqueued on
  * `stream` and the call returns without synchronising, except where stated.
  * Argument errors are detected on the host before anything is enqueued.
  * benes_route, benes_apply and benes_apply_ex do nothing but enqueue kernels and

@@ -29,6 +29,7 @@ constexpr size_t kAlign = 256;
 struct Workspace {
     void *own = nullptr;       // library-owned buffer
     size_t own_bytes = 0;
+    bool pooled = false;       // `own` came from the device's stream-ordered pool
     void *user = nullptr;      // caller-owned buffer (takes precedence)
     size_t user_bytes = 0;
 };
@@ -57,8 +58,46 @@ Options options() {
 
 inline size_t align_up(size_t v) { return (v + kAlign - 1) & ~(kAlign - 1); }
 
-// Returns a device scratch buffer of at least `bytes`.
-int get_workspace(size_t bytes, void **out) {
+bool pool_supported(int dev) {
+    static int cached[kMaxDevices] = {};           // 0 unknown, 1 yes, 2 no
+    if (!cached[dev]) {
+        int v = 0;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMemoryPoolsSupported, dev) != cudaSuccess) { cudaGetLastError(); v = 0; }
+        cached[dev] = v ? 1 : 2;
+    }
+    return cached[dev] == 1;
+}
+
+// Frees the library-owned buffer of `w` (g_mu held).  Stream-ordered on `s` if it came from the
+// pool and a stream is given; otherwise the device is synchronised first.
+int drop_own(Workspace &w, int dev, bool have_stream, cudaStream_t s) {
+    if (!w.own) return BENES_OK;
+    if (w.pooled && have_stream) {
+        BENES_CUDA_TRY(cudaFreeAsync(w.own, s));
+    } else {
+        BENES_CUDA_TRY(cudaDeviceSynchronize());
+        if (w.pooled) {
+            BENES_CUDA_TRY(cudaFreeAsync(w.own, nullptr));
+            BENES_CUDA_TRY(cudaStreamSynchronize(nullptr));
+            cudaMemPool_t pool = nullptr;
+            if (cudaDeviceGetDefaultMemPool(&pool, dev) == cudaSuccess && pool) cudaMemPoolTrimTo(pool, 0);
+            cudaGetLastError();
+        } else {
+            BENES_CUDA_TRY(cudaFree(w.own));
+        }
+    }
+    w.own = nullptr;
+    w.own_bytes = 0;
+    w.pooled = false;
+    return BENES_OK;
+}
+
+// Returns a device scratch buffer of at least `bytes` for work that is enqueued on `s`.  A
+// library-owned buffer that is too small is replaced in stream order (cudaFreeAsync +
+// cudaMallocAsync on `s`: no device-wide synchronisation; calls that share the workspace are
+// ordered by contract, so everything that used the old buffer precedes the free), or, on a
+// device without memory pools, after a device synchronisation.
+int get_workspace(size_t bytes, void **out, cudaStream_t s) {
     int dev = 0;
     BENES_CUDA_TRY(cudaGetDevice(&dev));
     if (dev < 0 || dev >= kMaxDevices) return BENES_ERR_CUDA;
@@ -70,18 +109,17 @@ int get_workspace(size_t bytes, void **out) {
         return BENES_OK;
     }
     if (bytes > w.own_bytes) {
-        if (w.own) {
-            BENES_CUDA_TRY(cudaDeviceSynchronize());
-            cudaFree(w.own);
-            w.own = nullptr;
-            w.own_bytes = 0;
-        }
-        if (cudaMalloc(&w.own, bytes) != cudaSuccess) {
+        const bool pool = pool_supported(dev);
+        int rc = drop_own(w, dev, pool, s);
+        if (rc) return rc;
+        const cudaError_t e = pool ? cudaMallocAsync(&w.own, bytes, s) : cudaMalloc(&w.own, bytes);
+        if (e != cudaSuccess) {
             cudaGetLastError();
             w.own = nullptr;
             return BENES_ERR_NOMEM;
         }
         w.own_bytes = bytes;
+        w.pooled = pool;
     }
     *out = w.own;
     return BENES_OK;
@@ -338,14 +376,7 @@ int benes_release_workspace(void) {
     BENES_CUDA_TRY(cudaGetDevice(&dev));
     if (dev < 0 || dev >= kMaxDevices) return BENES_ERR_CUDA;
     std::lock_guard<std::mutex> lk(g_mu);
-    Workspace &w = g_ws[dev];
-    if (w.own) {
-        BENES_CUDA_TRY(cudaDeviceSynchronize());
-        BENES_CUDA_TRY(cudaFree(w.own));
-        w.own = nullptr;
-        w.own_bytes = 0;
-    }
-    return BENES_OK;
+    return drop_own(g_ws[dev], dev, false, nullptr);
 }
 
 int benes_route(const uint32_t *perm, int log2n, int batch, uint32_t *switch_bits,
@@ -372,7 +403,7 @@ int benes_route(const uint32_t *perm, int log2n, int batch, uint32_t *switch_bit
         return launch_fused(perm, 0, size_t(batch) << n, n, switch_bits, n, s);
     }
     void *ws = nullptr;
-    int rc = get_workspace(route_ws_bytes(n, size_t(batch)), &ws);
+    int rc = get_workspace(route_ws_bytes(n, size_t(batch)), &ws, s);
     if (rc) return rc;
     const size_t chunk = level_chunk(n, size_t(batch), opt.chunk_log2);
     for (size_t b0 = 0; b0 < size_t(batch); b0 += chunk) {
@@ -394,7 +425,7 @@ int benes_apply_ex(const uint32_t *switch_bits, const void *in, void *out, int e
     const int stages = 2 * n - 1;
     void *ws = nullptr;
     if (n >= 2) {
-        int rc = get_workspace(apply_ws_bytes(elem_bytes, n, size_t(batch)), &ws);
+        int rc = get_workspace(apply_ws_bytes(elem_bytes, n, size_t(batch)), &ws, s);
         if (rc) return rc;
     }
     if (options().apply_fused) {
@@ -442,7 +473,7 @@ int benes_route_padded(const uint32_t *perm, size_t n_elems, int batch, uint32_t
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     const size_t inner = align_up(route_ws_bytes(n, size_t(batch)));
     void *ws = nullptr;
-    int rc = get_workspace(inner + align_up((size_t(batch) << n) * 4), &ws);
+    int rc = get_workspace(inner + align_up((size_t(batch) << n) * 4), &ws, s);
     if (rc) return rc;
     uint32_t *padded = reinterpret_cast<uint32_t *>(static_cast<char *>(ws) + inner);
     if ((rc = launch_pad_perm(perm, padded, n_elems, n, size_t(batch), s))) return rc;
@@ -459,7 +490,7 @@ int benes_apply_padded(const uint32_t *switch_bits, const void *in, void *out, i
     const size_t inner = align_up(apply_ws_bytes(elem_bytes, n, size_t(batch)));
     const size_t row_bytes = align_up((size_t(batch) << n) * size_t(elem_bytes));
     void *ws = nullptr;
-    int rc = get_workspace(inner + 2 * row_bytes, &ws);
+    int rc = get_workspace(inner + 2 * row_bytes, &ws, s);
     if (rc) return rc;
     char *pin = static_cast<char *>(ws) + inner, *pout = pin + row_bytes;
     if ((rc = launch_pad_rows(in, pin, elem_bytes, true, n_elems, n, size_t(batch), s))) return rc;
@@ -475,7 +506,7 @@ int benes_route_host(const uint32_t *perm_host, int log2n, int batch, uint32_t *
     const size_t bits_bytes = benes_switch_words(log2n, batch) * 4;
     const size_t inner = route_ws_bytes(log2n, size_t(batch));
     void *ws = nullptr;
-    int rc = get_workspace(align_up(inner) + align_up(perm_bytes) + align_up(bits_bytes), &ws);
+    int rc = get_workspace(align_up(inner) + align_up(perm_bytes) + align_up(bits_bytes), &ws, s);
     if (rc) return rc;
     char *base = static_cast<char *>(ws);
     uint32_t *d_perm = reinterpret_cast<uint32_t *>(base + align_up(inner));
@@ -522,7 +553,7 @@ int benes_apply_host(const uint32_t *switch_bits_host, const void *in_host, void
     const size_t bits_bytes = benes_switch_words(log2n, batch) * 4;
     const size_t inner = apply_ws_bytes(elem_bytes, log2n, size_t(batch));
     void *ws = nullptr;
-    int rc = get_workspace(align_up(inner) + 2 * align_up(data_bytes) + align_up(bits_bytes), &ws);
+    int rc = get_workspace(align_up(inner) + 2 * align_up(data_bytes) + align_up(bits_bytes), &ws, s);
     if (rc) return rc;
     char *base = static_cast<char *>(ws);
     char *d_in = base + align_up(inner);
@@ -596,7 +627,7 @@ int benes_route_apply_host(const uint32_t *perm_host, const void *in_host, void 
     const size_t route_ws = align_up(route_ws_bytes(n, size_t(batch)));
     const size_t apply_ws = align_up(apply_ws_bytes(elem_bytes, n, size_t(batch)));
     void *ws = nullptr;
-    int rc = get_workspace(route_ws + apply_ws + align_up(perm_bytes) + align_up(bits_bytes) + 2 * align_up(data_bytes), &ws);
+    int rc = get_workspace(route_ws + apply_ws + align_up(perm_bytes) + align_up(bits_bytes) + 2 * align_up(data_bytes), &ws, s);
     if (rc) return rc;
     char *base = static_cast<char *>(ws);
     char *scratch = base + route_ws;
@@ -651,7 +682,7 @@ int benes_validate_perm(const uint32_t *perm, int log2n, int batch, benes_stream
     const size_t total = size_t(batch) << log2n;
     const size_t seen_bytes = align_up(((total + 31) / 32) * 4);
     void *ws = nullptr;
-    int rc = get_workspace(seen_bytes + kAlign, &ws);
+    int rc = get_workspace(seen_bytes + kAlign, &ws, s);
     if (rc) return rc;
     uint32_t *seen = static_cast<uint32_t *>(ws);
     uint32_t *flag = reinterpret_cast<uint32_t *>(static_cast<char *>(ws) + seen_bytes);
