@@ -186,6 +186,26 @@ int benes_apply_host(const uint32_t *switch_bits_host, const void *in_host, void
 int benes_route_apply_host(const uint32_t *perm_host, const void *in_host, void *out_host, int elem_bytes,
                            int log2n, int batch, uint32_t *switch_bits_host, benes_stream_t stream);
 
+/*
+ * Plans: the same route (and, if `in` and `out` are given, the apply behind it)
+ * on the same buffers, many times.  benes_plan_create runs the work once on a
+ * stream of its own (synchronously), captures it into a CUDA graph and keeps a
+ * scratch buffer of its own for it (cudaMalloc; freed by benes_plan_destroy), so
+ * a plan is independent of the library workspace.  benes_plan_launch enqueues the
+ * whole graph on `stream` with one call: for inputs of up to about 2^22 elements,
+ * whose 2-50 dependent launches are short, that is 10-15 % faster than the
+ * launches themselves.  The plan reads whatever `perm` (and `in`) hold at launch
+ * time and is bound to the addresses, sizes and options it was created with; the
+ * buffers must outlive it.  Launches of one plan are ordered one after another.
+ * Not available while the per-kernel timing brackets are enabled.
+ *   in, out, elem_bytes : NULL, NULL, 0 for a route-only plan.
+ */
+typedef struct benes_plan benes_plan_t;
+int benes_plan_create(benes_plan_t **plan, const uint32_t *perm, int log2n, int batch, uint32_t *switch_bits,
+                      const void *in, void *out, int elem_bytes);
+int benes_plan_launch(const benes_plan_t *plan, benes_stream_t stream);
+int benes_plan_destroy(benes_plan_t *plan);
+
 /* Number of 32-bit words of switch_bits for (log2n, batch); 0 on bad arguments. */
 size_t benes_switch_words(int log2n, int batch);
 
@@ -267,6 +287,7 @@ unsigned long long benes_launch_count(void);
  */
 #define BENES_PROFILE_KINDS 12
 int benes_profile_enable(int on);
+int benes_profile_enabled(void);    /* 1 while the brackets are on */
 int benes_profile_reset(void);
 int benes_profile_read(int kind, unsigned long long *launches, double *milliseconds);
 /* The index-th timed group since the last reset, in launch order (one group per

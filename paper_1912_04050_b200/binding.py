@@ -47,6 +47,10 @@ SYMBOLS = {
     "benes_set_option": (_i, [_i, _i]),
     "benes_get_option": (_i, [_i]),
     "benes_launch_count": (ctypes.c_ulonglong, []),
+    "benes_plan_create": (_i, [ctypes.POINTER(_vp), _vp, _i, _i, _vp, _vp, _vp, _i]),
+    "benes_plan_launch": (_i, [_vp, _vp]),
+    "benes_plan_destroy": (_i, [_vp]),
+    "benes_profile_enabled": (_i, []),
     "benes_profile_enable": (_i, [_i]),
     "benes_profile_reset": (_i, []),
     "benes_profile_read": (_i, [_i, ctypes.POINTER(ctypes.c_ulonglong), ctypes.POINTER(ctypes.c_double)]),
@@ -208,6 +212,34 @@ def benes_route_apply_host(perm_host, in_host, out_host, elem_bytes: int, log2n:
     _check(load().benes_route_apply_host(_host_ptr(perm_host, "perm_host"), _host_ptr(in_host, "in_host"),
                                          _host_ptr(out_host, "out_host"), elem_bytes, log2n, batch, bits,
                                          _stream(stream)), "benes_route_apply_host")
+
+
+class Plan:
+    """A captured route (+ apply) on fixed buffers; launch() replays it with one call."""
+
+    def __init__(self, perm: torch.Tensor, log2n: int, batch: int, switch_bits: torch.Tensor,
+                 inp: torch.Tensor = None, out: torch.Tensor = None, elem_bytes: int = 0):
+        self._h = _vp(None)
+        self._keep = (perm, switch_bits, inp, out)          # the plan points into these
+        _check(load().benes_plan_create(ctypes.byref(self._h), _dev_ptr(perm, "perm"), log2n, batch,
+                                        _dev_ptr(switch_bits, "switch_bits"),
+                                        None if inp is None else _dev_ptr(inp, "in"),
+                                        None if out is None else _dev_ptr(out, "out"), elem_bytes),
+               "benes_plan_create")
+
+    def launch(self, stream=None) -> None:
+        _check(load().benes_plan_launch(self._h, _stream(stream)), "benes_plan_launch")
+
+    def destroy(self) -> None:
+        if self._h:
+            load().benes_plan_destroy(self._h)
+            self._h = _vp(None)
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
 
 
 def benes_set_workspace(buf, nbytes: int = 0) -> None:

@@ -4,6 +4,7 @@
 
 #include <cstdio>
 #include <mutex>
+#include <new>
 #include <vector>
 
 namespace benes {
@@ -379,11 +380,9 @@ int benes_release_workspace(void) {
     return drop_own(g_ws[dev], dev, false, nullptr);
 }
 
-int benes_route(const uint32_t *perm, int log2n, int batch, uint32_t *switch_bits,
-                benes_stream_t stream) {
-    if (!perm || !switch_bits || bad_shape(log2n, batch)) return BENES_ERR_BADARG;
-    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
-    const int n = log2n;
+// benes_route on a given scratch buffer (`ws` may be null when route_ws_bytes is 0)
+static int route_on(const uint32_t *perm, int n, int batch, uint32_t *switch_bits, char *ws, cudaStream_t s,
+                    const Options &opt) {
     if (n <= kFusedLog2M) {
         // whole permutations fit one CTA each
         const size_t max_ctas = size_t(1) << 30;
@@ -396,39 +395,30 @@ int benes_route(const uint32_t *perm, int log2n, int batch, uint32_t *switch_bit
         }
         return BENES_OK;
     }
-    const Options opt = options();
     if (n == kFusedLog2M + 1 && opt.cluster) {
         // whole permutations of 2^16, one cluster of two CTAs each
         ProfileScope ps(kFused, s);
         return launch_fused(perm, 0, size_t(batch) << n, n, switch_bits, n, s);
     }
-    void *ws = nullptr;
-    int rc = get_workspace(route_ws_bytes(n, size_t(batch)), &ws, s);
-    if (rc) return rc;
     const size_t chunk = level_chunk(n, size_t(batch), opt.chunk_log2);
     for (size_t b0 = 0; b0 < size_t(batch); b0 += chunk) {
         size_t nb = size_t(batch) - b0 < chunk ? size_t(batch) - b0 : chunk;
-        rc = route_levels(perm + (b0 << n), n, nb,
-                          switch_bits + b0 * size_t(2 * n - 1) * stage_words(n),
-                          static_cast<char *>(ws), s, opt);
+        int rc = route_levels(perm + (b0 << n), n, nb, switch_bits + b0 * size_t(2 * n - 1) * stage_words(n), ws,
+                              s, opt);
         if (rc) return rc;
     }
     return BENES_OK;
 }
 
-int benes_apply_ex(const uint32_t *switch_bits, const void *in, void *out, int elem_bytes,
-                   int log2n, int batch, benes_stream_t stream) {
-    if (!switch_bits || !in || !out || in == out || bad_shape(log2n, batch)) return BENES_ERR_BADARG;
-    if (elem_bytes != 4 && elem_bytes != 8) return BENES_ERR_BADARG;
-    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
-    const int n = log2n;
+static bool route_needs_ws(int n, const Options &opt) {
+    return n > kFusedLog2M && !(n == kFusedLog2M + 1 && opt.cluster);
+}
+
+// benes_apply_ex on a given scratch buffer of apply_ws_bytes
+static int apply_on(const uint32_t *switch_bits, const void *in, void *out, int elem_bytes, int n, int batch,
+                    void *ws, cudaStream_t s, const Options &opt) {
     const int stages = 2 * n - 1;
-    void *ws = nullptr;
-    if (n >= 2) {
-        int rc = get_workspace(apply_ws_bytes(elem_bytes, n, size_t(batch)), &ws, s);
-        if (rc) return rc;
-    }
-    if (options().apply_fused) {
+    if (opt.apply_fused) {
         ProfileScope ps(kApplyFused, s);
         return launch_apply_fused(switch_bits, in, out, ws, elem_bytes, n, size_t(batch), s);
     }
@@ -443,6 +433,32 @@ int benes_apply_ex(const uint32_t *switch_bits, const void *in, void *out, int e
         src = dst;
     }
     return BENES_OK;
+}
+
+int benes_route(const uint32_t *perm, int log2n, int batch, uint32_t *switch_bits,
+                benes_stream_t stream) {
+    if (!perm || !switch_bits || bad_shape(log2n, batch)) return BENES_ERR_BADARG;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    const Options opt = options();
+    void *ws = nullptr;
+    if (route_needs_ws(log2n, opt)) {
+        int rc = get_workspace(route_ws_bytes(log2n, size_t(batch)), &ws, s);
+        if (rc) return rc;
+    }
+    return route_on(perm, log2n, batch, switch_bits, static_cast<char *>(ws), s, opt);
+}
+
+int benes_apply_ex(const uint32_t *switch_bits, const void *in, void *out, int elem_bytes,
+                   int log2n, int batch, benes_stream_t stream) {
+    if (!switch_bits || !in || !out || in == out || bad_shape(log2n, batch)) return BENES_ERR_BADARG;
+    if (elem_bytes != 4 && elem_bytes != 8) return BENES_ERR_BADARG;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    void *ws = nullptr;
+    if (log2n >= 2) {
+        int rc = get_workspace(apply_ws_bytes(elem_bytes, log2n, size_t(batch)), &ws, s);
+        if (rc) return rc;
+    }
+    return apply_on(switch_bits, in, out, elem_bytes, log2n, batch, ws, s, options());
 }
 
 int benes_apply(const uint32_t *switch_bits, const void *in, void *out, int log2n, int batch,
@@ -674,6 +690,79 @@ int benes_route_apply_host(const uint32_t *perm_host, const void *in_host, void 
     cudaError_t e1 = cudaStreamSynchronize(s), e2 = cudaStreamSynchronize(hp->side), e3 = cudaStreamSynchronize(hp->back);
     if (rc) return rc;
     return (e1 == cudaSuccess && e2 == cudaSuccess && e3 == cudaSuccess) ? BENES_OK : BENES_ERR_CUDA;
+}
+
+struct benes_plan {
+    int dev = 0;
+    cudaGraph_t graph = nullptr;
+    cudaGraphExec_t exec = nullptr;
+    void *ws = nullptr;                   // the plan's own scratch: the captured launches point into it
+    unsigned long long launches = 0;
+};
+
+int benes_plan_destroy(benes_plan_t *plan) {
+    if (!plan) return BENES_OK;
+    if (plan->exec) cudaGraphExecDestroy(plan->exec);
+    if (plan->graph) cudaGraphDestroy(plan->graph);
+    if (plan->ws) cudaFree(plan->ws);
+    cudaGetLastError();
+    delete plan;
+    return BENES_OK;
+}
+
+int benes_plan_create(benes_plan_t **plan_out, const uint32_t *perm, int log2n, int batch, uint32_t *switch_bits,
+                      const void *in, void *out, int elem_bytes) {
+    if (!plan_out || !perm || !switch_bits || bad_shape(log2n, batch)) return BENES_ERR_BADARG;
+    const bool with_apply = in != nullptr || out != nullptr;
+    if (with_apply && (!in || !out || in == out || (elem_bytes != 4 && elem_bytes != 8))) return BENES_ERR_BADARG;
+    if (benes_profile_enabled()) return BENES_ERR_BADARG;      // event brackets cannot live inside a graph
+    *plan_out = nullptr;
+    const Options opt = options();
+    const int n = log2n;
+    benes_plan *p = new (std::nothrow) benes_plan;
+    if (!p) return BENES_ERR_NOMEM;
+    cudaStream_t cap = nullptr;
+    int rc = BENES_OK;
+    auto fail = [&](int code) {
+        if (cap) cudaStreamDestroy(cap);
+        benes_plan_destroy(p);
+        cudaGetLastError();
+        return code;
+    };
+    if (cudaGetDevice(&p->dev) != cudaSuccess) return fail(BENES_ERR_CUDA);
+    const size_t route_ws = route_needs_ws(n, opt) ? align_up(route_ws_bytes(n, size_t(batch))) : 0;
+    const size_t apply_ws = with_apply ? align_up(apply_ws_bytes(elem_bytes, n, size_t(batch))) : 0;
+    if (route_ws + apply_ws) {
+        if (cudaMalloc(&p->ws, route_ws + apply_ws) != cudaSuccess) return fail(BENES_ERR_NOMEM);
+    }
+    char *ws = static_cast<char *>(p->ws);
+    if (cudaStreamCreateWithFlags(&cap, cudaStreamNonBlocking) != cudaSuccess) return fail(BENES_ERR_CUDA);
+    auto enqueue = [&]() -> int {
+        int r = route_on(perm, n, batch, switch_bits, ws, cap, opt);
+        if (!r && with_apply) r = apply_on(switch_bits, in, out, elem_bytes, n, batch, ws + route_ws, cap, opt);
+        return r;
+    };
+    // once plainly (every kernel's attributes get set, and the buffers are checked by use), then captured
+    if ((rc = enqueue())) return fail(rc);
+    if (cudaStreamSynchronize(cap) != cudaSuccess) return fail(BENES_ERR_CUDA);
+    const unsigned long long l0 = g_launches;
+    if (cudaStreamBeginCapture(cap, cudaStreamCaptureModeThreadLocal) != cudaSuccess) return fail(BENES_ERR_CUDA);
+    rc = enqueue();
+    const cudaError_t e = cudaStreamEndCapture(cap, &p->graph);
+    if (rc) return fail(rc);
+    if (e != cudaSuccess || !p->graph) return fail(BENES_ERR_CUDA);
+    p->launches = g_launches - l0;
+    if (cudaGraphInstantiate(&p->exec, p->graph, 0) != cudaSuccess) return fail(BENES_ERR_CUDA);
+    cudaStreamDestroy(cap);
+    *plan_out = p;
+    return BENES_OK;
+}
+
+int benes_plan_launch(const benes_plan_t *plan, benes_stream_t stream) {
+    if (!plan || !plan->exec) return BENES_ERR_BADARG;
+    BENES_CUDA_TRY(cudaGraphLaunch(plan->exec, reinterpret_cast<cudaStream_t>(stream)));
+    g_launches += plan->launches;
+    return BENES_OK;
 }
 
 int benes_validate_perm(const uint32_t *perm, int log2n, int batch, benes_stream_t stream) {

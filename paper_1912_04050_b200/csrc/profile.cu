@@ -69,6 +69,11 @@ int benes_profile_enable(int on) {
     return BENES_OK;
 }
 
+int benes_profile_enabled(void) {
+    std::lock_guard<std::mutex> lk(g_pmu);
+    return g_enabled ? 1 : 0;
+}
+
 int benes_profile_reset(void) {
     std::lock_guard<std::mutex> lk(g_pmu);
     for (Span &sp : g_spans) {

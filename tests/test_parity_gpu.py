@@ -583,6 +583,41 @@ def test_route_and_apply_replayed_from_a_cuda_graph(n, batch):
         assert np.array_equal(host(out, np.uint64).reshape(x.shape), np.take_along_axis(x, perm.astype(np.int64), axis=1))
 
 
+@pytest.mark.parametrize("n,batch,with_apply", [(8, 100, True), (12, 4, True), (16, 3, True), (18, 1, False),
+                                                (20, 1, True)])
+def test_plans_replay_the_route_on_fixed_buffers(n, batch, with_apply):
+    """benes_plan_create captures route (+ apply) once; every launch reads the buffers' current
+    contents.  Two plans coexist (each has its own scratch), and ordinary calls in between do
+    not disturb them."""
+    perms = [inputs.random_perm_batch(n, batch, seed0=700 + n + 50 * k) for k in range(3)]
+    x = inputs.payload_u64(batch << n, 3).reshape(batch, -1)
+    d_perm, d_x = dev(perms[0]), dev(x)
+    bits = torch.empty(binding.benes_switch_words(n, batch), dtype=torch.int32, device="cuda")
+    out = torch.empty_like(d_x)
+    plan = binding.Plan(d_perm, n, batch, bits, d_x, out, 8) if with_apply else binding.Plan(d_perm, n, batch, bits)
+    other_perm = dev(perms[1])
+    other_bits = torch.empty_like(bits)
+    other = binding.Plan(other_perm, n, batch, other_bits)
+    before = binding.benes_launch_count()
+    shape = (batch, 2 * n - 1, max(1, (1 << n) // 64))
+    for k in (1, 2, 0, 2):
+        d_perm.copy_(dev(perms[k]))
+        bits.fill_(-1)
+        out.fill_(-1)
+        plan.launch()
+        other.launch()
+        gpu_route(perms[(k + 1) % 3], n)                       # an ordinary call in between (library workspace)
+        torch.cuda.synchronize()
+        assert np.array_equal(host(bits, np.uint32).reshape(shape), oracle.route(perms[k], n))
+        assert np.array_equal(host(other_bits, np.uint32).reshape(shape), oracle.route(perms[1], n))
+        if with_apply:
+            assert np.array_equal(host(out, np.uint64).reshape(x.shape),
+                                  np.take_along_axis(x, perms[k].astype(np.int64), axis=1))
+    assert binding.benes_launch_count() > before                # replayed launches are counted too
+    plan.destroy()
+    other.destroy()
+
+
 def test_launch_counter_counts():
     n = 17
     before = binding.benes_launch_count()
