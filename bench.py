@@ -691,6 +691,7 @@ def run_gpu(args):
                 # what the DRAM actually moved for this kernel (ncu counters of the same workload)
                 roofline["dram_gbs"] = traffic / per_launch_s / 1e9
                 roofline["dram_frac"] = traffic / per_launch_s / 1e9 / peak
+                roofline["dram_frac_of_nominal_8tbs"] = traffic / per_launch_s / 1e9 / 8000.0
             if top == "walk" and per_level.get("walk") and probe:
                 # The walk is a chain of dependent random accesses: per switch one record visit
                 # (load + claim) and one 4-byte inverse entry.  Level 0 is the launch whose block
